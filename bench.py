@@ -1,0 +1,352 @@
+#!/usr/bin/env python
+"""Benchmark of the hybrid-attention forward pass (one layer = one step).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload wan81]
+
+Prints ONE JSON line.  A step is one pass of the whole hot path (K pass -> state reduction ->
+Q pass) over one synthetic layer input already resident in HBM; `e2e` is the same step through
+the host-buffer entry point with the host<->device copies inside the timed region.  With
+N > 1 (torchrun) every rank runs its own layer input (independent batches, no collective in
+the data path) and the value is the aggregate over ranks.  `--impl reference` times the
+float64 CPU oracle on the host cores instead (a deliberately slow baseline).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "hybrid-attn fwd tokens/s per layer at N=32760 (12x128 heads); % of bf16 tensor peak"
+
+# DRAM bytes of one Q-pass launch at the wan81 workload (dram__bytes_read.sum + dram__bytes_write.sum
+# from the ncu capture summarised in profiles/); None until a capture exists.
+QPASS_DRAM_TRAFFIC_BYTES = {}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def flops_per_layer(wl, n_s):
+    """Algorithmic FLOPs of one layer (all heads), split per kernel."""
+    N, d, F = wl.N, wl.d, wl.F
+    n_l = N - n_s
+    heads = wl.B * wl.H
+    kpass = (2 * d * F * n_l + 2 * n_l * F * (d + 1)) if n_l > 0 else 0
+    qpass = 4 * N * n_s * d + ((2 * N * d * F + 2 * N * F * (d + 1)) if n_l > 0 else 0)
+    return {"kpass": heads * kpass, "qpass": heads * qpass, "total": heads * (kpass + qpass)}
+
+
+def bytes_per_layer(wl):
+    """Algorithmic HBM bytes of one layer: q, k, v read once, out written once."""
+    return 4 * wl.B * wl.H * wl.N * wl.d * 2
+
+
+class ClockSampler:
+    """Samples SM clock and clock-event reasons of one GPU through NVML in a background thread."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.period, self.samples, self._stop = period_s, [], threading.Event()
+        self.max_mhz, self.ok = None, False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            idx = index
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            if vis:
+                try:
+                    idx = int(vis.split(",")[index])
+                except ValueError:
+                    idx = index
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+        self.thread = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.samples.append((mhz, reasons))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.ok:
+            self.thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self.ok and self.thread.is_alive():
+            self.thread.join(timeout=1.0)
+
+    def summary(self):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"], "samples": 0}
+        bits = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+                0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown", 0x10: "sync_boost"}
+        seen = set()
+        for _, r in self.samples:
+            for b, name in bits.items():
+                if r & b:
+                    seen.add(name)
+        return {"sm_mhz": statistics.median(m for m, _ in self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(seen), "samples": len(self.samples)}
+
+
+def cpu_oracle_rate(wl, data64, mask, budget_s, heads=1, rows0=256):
+    """Times the float64 oracle on a bounded sample and extrapolates to tokens/s of a full layer.
+
+    Sample: `heads` heads; the linear state over all tokens (timed alone), then the full operator on
+    `rows` query rows.  Per-row cost = (t_rows - t_state) / rows; a full layer costs
+    H * (t_state + N * t_row) per batch element."""
+    from oracle import hybrid_attention as O
+    import numpy as np
+    n_l = int((~mask).sum())
+    q, k, v = data64["q"][0], data64["k"][0], data64["v"][0]
+
+    def one(rows):
+        t_state = t_rows = 0.0
+        for h in range(heads):
+            if n_l > 0:
+                t0 = time.perf_counter()
+                O.linear_state(k[h], v[h], data64["wk"][h], mask, wl.degree)
+                t_state += time.perf_counter() - t0
+            t0 = time.perf_counter()
+            O.hybrid_attention_head(q[h], k[h], v[h], data64["wq"][h], data64["wk"][h], mask, None,
+                                    O.STAB_PAPER, wl.degree, rows=rows)
+            t_rows += time.perf_counter() - t0
+        return t_state / heads, t_rows / heads
+
+    rows = np.arange(min(rows0, wl.N))
+    ts, tr = one(rows)
+    t_row = max(tr - ts, 1e-9) / len(rows)
+    # grow the sample towards the budget
+    want = int(min(wl.N, max(len(rows), (budget_s / heads - 2 * ts) / t_row)))
+    if want > 2 * len(rows):
+        rows = np.arange(want)
+        ts, tr = one(rows)
+        t_row = max(tr - ts, 1e-9) / len(rows)
+    layer_s = wl.H * (ts + wl.N * t_row)            # per batch element
+    return {"tokens_per_s": wl.N / layer_s, "rows": int(len(rows)), "heads": heads,
+            "t_state_s": ts, "t_rows_s": tr, "step_s": heads * (ts + tr)}
+
+
+def run_reference(args, wl):
+    """The oracle, as it stands, on the host cores: K timed steps of a bounded sample each."""
+    import numpy as np
+    from oracle import hybrid_attention as O
+    from paper_2509_24899_b200 import workloads as W
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    cores = os.cpu_count() or 1
+    data64 = {k: W.bf16_bits_to_f64(v) for k, v in W.generate(wl, heads=1).items()}
+    mask = O.softmax_token_mask(wl.grid, wl.block, wl.rate)
+    total = args.steps + args.warmup
+    budget = max(0.05, min(2.0, 150.0 / total))
+    vals, step_s, last = [], [], None
+    for i in range(total):
+        r = cpu_oracle_rate(wl, data64, mask, budget_s=budget, heads=1, rows0=128)
+        if i >= args.warmup:
+            vals.append(r["tokens_per_s"])
+            step_s.append(r["step_s"])
+            last = r
+    value = statistics.mean(vals)                      # one host, whatever N is
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wl.B * wl.N / value,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "d": wl.d, "F": wl.F,
+                   "rate": wl.rate, "n_softmax": int(mask.sum())},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                         "sample": "per step: 1 head, linear state over all tokens + %d query rows against all "
+                                   "keys; extrapolated to H heads x N rows" % last["rows"]},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def run_ours(args, wl):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2509_24899_b200 import HybridAttention, binding, workloads as W
+    import dataclasses
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # every rank draws its own layer input (independent batches: weak scaling, no exchange step)
+    wl_r = dataclasses.replace(wl, seed=wl.seed + rank)
+    data = W.generate(wl_r)
+    to_dev = lambda b: torch.from_numpy(b.view(np.int16)).cuda().view(torch.bfloat16)
+    dev = {k: to_dev(v) for k, v in data.items()}
+    path = {"tensor": binding.AS_PATH_TENSOR, "simt": binding.AS_PATH_SIMT}[args.path]
+    op = HybridAttention.from_workload(wl_r, kernel_path=path)
+    out = torch.empty_like(dev["q"])
+    stream = torch.cuda.current_stream()
+    step = lambda: op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], out=out, stream=stream)
+
+    sampler = ClockSampler(local)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    assert op.last_status() == 0, "device time-out during warm-up"
+
+    binding.as_hybrid_attn_profile_enable(op.handle, True)
+    launches0 = binding.as_hybrid_attn_launch_count(op.handle)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = binding.as_hybrid_attn_launch_count(op.handle) - launches0
+    kms, kcnt = binding.as_hybrid_attn_profile_read(op.handle)
+    binding.as_hybrid_attn_profile_enable(op.handle, False)
+    status = op.last_status()
+
+    # end to end: host buffers in, host buffer out, copies inside the timed region
+    host = {k: torch.from_numpy(data[k].view(np.int16)).pin_memory() for k in ("q", "k", "v")}
+    out_host = torch.empty_like(host["q"]).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(2):
+        op.forward_host(host["q"], host["k"], host["v"], dev["wq"], dev["wk"], out_host, stream=stream)
+    barrier()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        op.forward_host(host["q"], host["k"], host["v"], dev["wq"], dev["wk"], out_host, stream=stream)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    sampler.stop()
+
+    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, e2e_ms = t.tolist()
+    tokens = wl.B * wl.N * world
+    value = tokens * args.steps / (ms * 1e-3)
+    e2e_value = tokens * e2e_steps / (e2e_ms * 1e-3)
+
+    rc = 0
+    if rank == 0:
+        peaks = _peaks()
+        n_s = op.n_softmax
+        fl = flops_per_layer(wl, n_s)
+        q_launches = max(kcnt[binding.AS_KERNEL_QPASS], 1)
+        q_ms = kms[binding.AS_KERNEL_QPASS] / q_launches
+        k_ms = kms[binding.AS_KERNEL_KPASS] / max(kcnt[binding.AS_KERNEL_KPASS], 1)
+        r_ms = kms[binding.AS_KERNEL_REDUCE] / max(kcnt[binding.AS_KERNEL_REDUCE], 1)
+        if n_s > 0:
+            achieved = fl["qpass"] / (q_ms * 1e-3) / 1e12
+            roof = {"bound": "tensor", "kernel": "qpass", "achieved": achieved, "peak": peaks["bf16_tflops"],
+                    "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                    "traffic": QPASS_DRAM_TRAFFIC_BYTES.get(wl.name),
+                    "peak_source": "%s burst bf16 (sustained %s)" % (peaks["source"], peaks["bf16_tflops_sustained"]),
+                    "frac_of_nominal_2250": achieved / 2250.0, "avg_launch_ms": q_ms,
+                    "flops_per_launch": fl["qpass"]}
+        else:       # rate 0: the whole layer is bound by reading q, k, v and writing out
+            gbs = bytes_per_layer(wl) / ((k_ms + r_ms + q_ms) * 1e-3) / 1e9
+            roof = {"bound": "hbm", "kernel": "kpass+qpass", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                    "peak_source": peaks["source"]}
+        # CPU baseline: the oracle on this machine's host cores, bounded sample
+        from oracle import hybrid_attention as O
+        cores = os.cpu_count() or 1
+        d1 = {k: W.bf16_bits_to_f64(v[:, :1] if k in ("q", "k", "v") else v[:1]) for k, v in data.items()}
+        mask = O.softmax_token_mask(wl.grid, wl.block, wl.rate)
+        cb = cpu_oracle_rate(wl, d1, mask, budget_s=15.0, heads=1)
+        clocks = sampler.summary()
+        line = {
+            "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "d": wl.d, "F": wl.F,
+                       "rate": wl.rate, "n_softmax": n_s, "stab_mode": "paper", "kernel_path": args.path,
+                       "l2": "q,k,v,out of a step total %.0f MB > 126 MB L2" % (bytes_per_layer(wl) / 1e6),
+                       "parallelism": "dp%d (independent layer inputs per rank)" % world},
+            "tflops": fl["total"] * args.steps / (ms * 1e-3) / 1e12 * 1.0,
+            "kernel_ms": {"kpass": k_ms, "reduce": r_ms, "qpass": q_ms},
+            "roofline": roof,
+            "cpu_baseline": {"value": cb["tokens_per_s"], "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                             "sample": "1 head: linear state over all tokens + %d query rows against all keys; "
+                                       "extrapolated to %d heads x %d rows" % (cb["rows"], wl.H, wl.N)},
+            "e2e": {"value": e2e_value, "unit": "tokens/s",
+                    "h2d_bytes_per_step": 3 * wl.B * wl.H * wl.N * wl.d * 2,
+                    "d2h_bytes_per_step": wl.B * wl.H * wl.N * wl.d * 2, "steps": e2e_steps},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "device_status": status,
+        }
+        print(json.dumps(line))
+        if status != 0:
+            rc = 1
+    if world > 1:
+        dist.destroy_process_group()
+    return rc
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="wan81",
+                    help="tiny | wan17 | wan81 | wan161cfg | stack:<layer>")
+    ap.add_argument("--path", default="tensor", choices=["tensor", "simt"],
+                    help="kernel path: tcgen05 tensor-core kernels (default) or the fp32 CUDA-core check path")
+    args = ap.parse_args()
+    from paper_2509_24899_b200 import workloads as W
+    if args.workload.startswith("stack:"):
+        wl = W.stack_layer(int(args.workload.split(":")[1]))
+    else:
+        wl = W.CONFIGS[args.workload]
+    if args.impl == "reference":
+        return run_reference(args, wl)
+    return run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

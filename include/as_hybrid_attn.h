@@ -1,0 +1,173 @@
+/*
+ * as_hybrid_attn.h - C ABI of the hybrid-attention forward pass for NVIDIA B200 (sm_100a).
+ *
+ * The operator is the hybrid attention of "Attention Surgery" (arXiv 2509.24899), section
+ * "Hybrid Attention": for every query i
+ *
+ *        sum_{j in T_S} exp(q_i.k_j * scale - c_i) v_j  +  lambda_i * phi_q(q_i) S
+ *  y_i = -----------------------------------------------------------------------------
+ *        sum_{j in T_S} exp(q_i.k_j * scale - c_i)      +  lambda_i * phi_q(q_i) . z
+ *
+ *  S = sum_{j in T_L} phi_k(k_j)^T v_j   [F x d],      z = sum_{j in T_L} phi_k(k_j)   [F],
+ *  c_i = max_{j in T_S} q_i.k_j * scale,
+ *
+ * where the tokens T = {0..N-1} are split into softmax tokens T_S and linear tokens
+ * T_L = T \ T_S by the hybrid rate R (same section: every R-th token is a softmax token), and
+ * phi_q, phi_k are the learned polynomial feature maps of "Characterization of phi".
+ * Rate 1 is plain softmax attention (Eq. 2); rate 0 is normalised linear attention (the
+ * kernelised form in "Preliminaries: Linear Attention").
+ *
+ * Conventions
+ *   - All tensor pointers are DEVICE pointers unless a parameter says "host".
+ *   - q, k, v, out: [B, H, N, d] bf16, contiguous, base address 16-byte aligned.
+ *   - The caller owns every buffer and the CUDA stream; the library owns only the handle.
+ *   - Every function returns a status; nothing aborts, and no kernel traps.  On error the
+ *     out-parameters are left untouched.
+ *   - `forward` is asynchronous on the given stream, allocates nothing and does not
+ *     synchronise.  One handle may be used concurrently only with distinct workspaces.
+ */
+#ifndef AS_HYBRID_ATTN_H_
+#define AS_HYBRID_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define AS_API __attribute__((visibility("default")))
+#else
+#define AS_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct as_hybrid_attn_s* as_hybrid_attn_t;   /* opaque, library-owned */
+
+typedef enum {
+  AS_OK = 0,
+  AS_ERR_INVALID_ARG = 1,     /* NULL pointer, bad shape, misaligned buffer, inconsistent sizes   */
+  AS_ERR_UNSUPPORTED = 2,     /* valid request that this build has no kernel for                   */
+  AS_ERR_ARCH = 3,            /* current device is not compute capability 10.x                      */
+  AS_ERR_ALLOC = 4,           /* host or device allocation failed in create                        */
+  AS_ERR_WORKSPACE = 5,       /* workspace NULL, misaligned or smaller than workspace_bytes         */
+  AS_ERR_CUDA = 6,            /* a CUDA runtime/driver call failed                                  */
+  AS_ERR_DEVICE_TIMEOUT = 7   /* a bounded wait inside a kernel ran out (see last_status)           */
+} as_status_t;
+
+/* Stabiliser handling (the paper subtracts c_i only inside the softmax exponentials):
+ *   AS_STAB_PAPER  lambda_i = 1            - the equation exactly as printed;
+ *   AS_STAB_EXACT  lambda_i = exp(-c_i)    - weights exp(s_ij) beside phi_q.phi_k, independent of c_i. */
+enum { AS_STAB_PAPER = 0, AS_STAB_EXACT = 1 };
+
+/* Activation of the feature map's embedding layers. */
+enum { AS_ACT_RELU = 0 };
+
+/* Kernel path.  AS_PATH_TENSOR: tcgen05/TMEM/TMA kernels (the product path).
+ * AS_PATH_SIMT: plain fp32 CUDA-core kernels kept as an on-device cross-check. */
+enum { AS_PATH_TENSOR = 0, AS_PATH_SIMT = 1 };
+
+/* Kernel classes reported by the profiling calls. */
+enum { AS_KERNEL_KPASS = 0, AS_KERNEL_REDUCE = 1, AS_KERNEL_QPASS = 2, AS_NUM_KERNELS = 3 };
+
+typedef struct {
+  uint32_t struct_size;            /* sizeof(as_hybrid_attn_desc_t), for ABI versioning            */
+  int32_t  B, H, N, d;             /* batch, heads, tokens, head dim; d in {64, 128}               */
+  int32_t  grid_t, grid_h, grid_w; /* latent grid, product == N; tokens row-major, w fastest       */
+  int32_t  blk_t, blk_h, blk_w;    /* spatial block (clipped at the grid border).  Inside each
+                                      block the token with 0-based raster index l is a softmax
+                                      token iff l mod R == 0.  A block equal to the grid gives the
+                                      paper's 1-D rule  T_S = { i : i mod R = 1 }  (1-indexed).     */
+  int32_t  rate_den;               /* R: 1 = every token softmax, 0 = none, else rate 1/R          */
+  const int32_t* softmax_idx;      /* optional HOST pointer to an explicit sorted, unique T_S;
+                                      NULL selects the rule above                                   */
+  int32_t  n_softmax;              /* length of softmax_idx (ignored when it is NULL)              */
+  int32_t  phi_dim;                /* F: output width of the feature map, in {64, 128}, == P * D'   */
+  int32_t  phi_layers;             /* embedding-network depth; 1 is supported                       */
+  int32_t  phi_hidden;             /* hidden width when phi_layers == 2 (unused otherwise)          */
+  int32_t  poly_degree;            /* P: part p (1-based) of the activation is raised to power p;
+                                      1 or 2 is supported                                            */
+  int32_t  phi_act;                /* AS_ACT_RELU                                                   */
+  float    softmax_scale;          /* 0 selects 1/sqrt(d)                                           */
+  int32_t  stab_mode;              /* AS_STAB_PAPER | AS_STAB_EXACT                                 */
+  int32_t  kernel_path;            /* AS_PATH_TENSOR | AS_PATH_SIMT                                 */
+} as_hybrid_attn_desc_t;
+
+/* Feature-map weights, DEVICE pointers, bf16, row-major with the output feature as the slow
+ * index: w*1 is [H, F, d] when phi_layers == 1.  Biases and second layers must be NULL in this
+ * build.  phi(x) = [a_1, a_2^2] with a = ReLU(W x) split into P contiguous parts. */
+typedef struct {
+  const void *wq1, *bq1, *wq2, *bq2;
+  const void *wk1, *bk1, *wk2, *bk2;
+} as_phi_weights_t;
+
+/* Creates a handle for one layer geometry on the CURRENT device: validates the descriptor,
+ * builds the token split on the host (section "Hybrid Attention", token rule) and uploads the
+ * index tables.  Returns AS_ERR_ARCH when the current device is not sm_100. */
+AS_API as_status_t as_hybrid_attn_create(const as_hybrid_attn_desc_t* desc, as_hybrid_attn_t* out);
+
+/* Frees the handle and its device tables.  NULL is a no-op. */
+AS_API as_status_t as_hybrid_attn_destroy(as_hybrid_attn_t h);
+
+/* Bytes of scratch `forward` needs (compacted softmax K/V, partial and final linear state). */
+AS_API as_status_t as_hybrid_attn_workspace_bytes(as_hybrid_attn_t h, size_t* bytes);
+
+/* Bytes of scratch `forward_host` needs: the above plus device staging for q, k, v and out. */
+AS_API as_status_t as_hybrid_attn_workspace_bytes_host(as_hybrid_attn_t h, size_t* bytes);
+
+/* The hybrid attention forward pass (equation above; hybrid equation of the paper).
+ *   q, k, v   [B,H,N,d] bf16 device, read only
+ *   w         feature-map weights (may be NULL only when rate_den == 1)
+ *   out       [B,H,N,d] bf16 device, written
+ *   aux       optional [B,H,N,3] fp32 device: (c_i, den_S, den_L) with
+ *             den_S = sum_{T_S} exp(s_ij - c_i), den_L = phi_q(q_i).z (before lambda_i); NULL to skip
+ *   workspace device scratch, 256-byte aligned, >= workspace_bytes; contents are overwritten
+ *   cuda_stream  a cudaStream_t (NULL = default stream)
+ * Enqueues its kernels and returns; errors found on the host are returned at once, a device
+ * time-out is reported later by as_hybrid_attn_last_status. */
+AS_API as_status_t as_hybrid_attn_forward(as_hybrid_attn_t h, const void* q, const void* k, const void* v,
+                                   const as_phi_weights_t* w, void* out, float* aux,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Same operation with HOST q, k, v and out buffers (pinned memory keeps the copies asynchronous):
+ * copies q, k, v to staging space in the workspace, runs forward, copies the result back, all on
+ * the stream.  The weights stay device pointers.  workspace >= workspace_bytes_host. */
+AS_API as_status_t as_hybrid_attn_forward_host(as_hybrid_attn_t h, const void* q_host, const void* k_host,
+                                        const void* v_host, const as_phi_weights_t* w,
+                                        void* out_host, void* workspace, size_t workspace_bytes,
+                                        void* cuda_stream);
+
+/* Copies the linear state left in `workspace` by the last forward on `cuda_stream`:
+ * S_out [B,H,F,d] fp32 and z_out [B,H,F] fp32 (device pointers; either may be NULL).
+ * S = sum_{T_L} phi_k(k_j)^T v_j, z = sum_{T_L} phi_k(k_j) ("Preliminaries: Linear Attention":
+ * the two sums that do not depend on the query).  AS_ERR_INVALID_ARG when rate_den == 1. */
+AS_API as_status_t as_hybrid_attn_linear_state(as_hybrid_attn_t h, const void* workspace,
+                                        float* S_out, float* z_out, void* cuda_stream);
+
+/* Number of softmax tokens |T_S| and, optionally, their sorted indices (HOST buffer of
+ * `capacity` int32; NULL to skip).  Token rule of section "Hybrid Attention". */
+AS_API as_status_t as_hybrid_attn_softmax_tokens(as_hybrid_attn_t h, int32_t* count,
+                                          int32_t* idx_host, int32_t capacity);
+
+/* Synchronises `cuda_stream`, then reads and clears the handle's device status word.
+ * AS_OK, AS_ERR_DEVICE_TIMEOUT (a bounded barrier wait in a kernel expired; outputs of that
+ * forward are undefined but the context stays usable) or AS_ERR_CUDA. */
+AS_API as_status_t as_hybrid_attn_last_status(as_hybrid_attn_t h, void* cuda_stream);
+
+/* Profiling aid: after `profile_enable(h, 1)` every kernel launch is bracketed by CUDA events on
+ * the launching stream.  `profile_read` synchronises those events, adds the elapsed device time
+ * per kernel class into ms[AS_NUM_KERNELS] and the launch counts into launches[AS_NUM_KERNELS],
+ * and resets the counters.  At most 1024 launches are kept between two reads. */
+AS_API as_status_t as_hybrid_attn_profile_enable(as_hybrid_attn_t h, int32_t enable);
+AS_API as_status_t as_hybrid_attn_profile_read(as_hybrid_attn_t h, float* ms, int32_t* launches);
+
+/* Total number of kernels this handle has launched since create. */
+AS_API as_status_t as_hybrid_attn_launch_count(as_hybrid_attn_t h, uint64_t* count);
+
+/* Static description of a status code. */
+AS_API const char* as_status_string(as_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* AS_HYBRID_ATTN_H_ */

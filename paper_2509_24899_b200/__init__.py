@@ -1,0 +1,104 @@
+"""B200-native hybrid attention forward (Attention Surgery, arXiv 2509.24899).
+
+`binding` mirrors the C ABI one to one; `HybridAttention` is a small convenience wrapper that
+lets PyTorch own the device memory and the stream.  All arithmetic runs in the CUDA library.
+"""
+from __future__ import annotations
+
+from . import binding
+from .binding import (AS_PATH_SIMT, AS_PATH_TENSOR, AS_STAB_EXACT, AS_STAB_PAPER, AsError)
+
+__all__ = ["binding", "HybridAttention", "AS_PATH_SIMT", "AS_PATH_TENSOR", "AS_STAB_EXACT",
+           "AS_STAB_PAPER", "AsError"]
+
+
+class HybridAttention:
+    """One layer geometry bound to the current CUDA device.
+
+    q, k, v: torch.bfloat16 CUDA tensors [B, H, N, d]; wq, wk: bfloat16 [H, F, d].
+    """
+
+    def __init__(self, B, H, N, d, grid, block, rate, phi_dim=None, poly_degree=2, softmax_scale=0.0,
+                 stab_mode=AS_STAB_PAPER, kernel_path=AS_PATH_TENSOR, softmax_idx=None):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("HybridAttention needs a CUDA device; there is no CPU fallback")
+        self.shape = (B, H, N, d)
+        self.F = d if phi_dim is None else phi_dim
+        self.rate = rate
+        self._desc = binding.make_desc(B, H, N, d, grid, block, rate, phi_dim, poly_degree, softmax_scale,
+                                       stab_mode, kernel_path, softmax_idx)
+        self._h = binding.as_hybrid_attn_create(self._desc)
+        self.workspace_bytes = binding.as_hybrid_attn_workspace_bytes(self._h)
+        self.workspace_bytes_host = binding.as_hybrid_attn_workspace_bytes_host(self._h)
+        self.n_softmax, _ = binding.as_hybrid_attn_softmax_tokens(self._h, want_indices=False)
+        self._ws = None
+
+    @classmethod
+    def from_workload(cls, wl, **kw):
+        return cls(wl.B, wl.H, wl.N, wl.d, wl.grid, wl.block, wl.rate, phi_dim=wl.F,
+                   poly_degree=wl.degree, **kw)
+
+    @property
+    def handle(self):
+        return self._h
+
+    def workspace(self, host: bool = False):
+        import torch
+        need = self.workspace_bytes_host if host else self.workspace_bytes
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        return self._ws
+
+    def softmax_indices(self):
+        return binding.as_hybrid_attn_softmax_tokens(self._h)[1]
+
+    def forward(self, q, k, v, wq=None, wk=None, out=None, aux=None, stream=None):
+        import torch
+        if out is None:
+            out = torch.empty_like(q)
+        ws = self.workspace()
+        st = torch.cuda.current_stream() if stream is None else stream
+        binding.as_hybrid_attn_forward(
+            self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(),
+            0 if wq is None else wq.data_ptr(), 0 if wk is None else wk.data_ptr(),
+            out.data_ptr(), 0 if aux is None else aux.data_ptr(), ws.data_ptr(), ws.numel(), st.cuda_stream)
+        return out
+
+    def forward_host(self, q_host, k_host, v_host, wq, wk, out_host, stream=None):
+        """q_host, k_host, v_host, out_host: pinned CPU tensors; wq, wk: device tensors."""
+        import torch
+        ws = self.workspace(host=True)
+        st = torch.cuda.current_stream() if stream is None else stream
+        binding.as_hybrid_attn_forward_host(
+            self._h, q_host.data_ptr(), k_host.data_ptr(), v_host.data_ptr(),
+            0 if wq is None else wq.data_ptr(), 0 if wk is None else wk.data_ptr(),
+            out_host.data_ptr(), ws.data_ptr(), ws.numel(), st.cuda_stream)
+        return out_host
+
+    def linear_state(self, stream=None):
+        """(S [B,H,F,d], z [B,H,F]) fp32 as left in the workspace by the last forward."""
+        import torch
+        B, H, N, d = self.shape
+        S = torch.empty(B, H, self.F, d, dtype=torch.float32, device="cuda")
+        z = torch.empty(B, H, self.F, dtype=torch.float32, device="cuda")
+        st = torch.cuda.current_stream() if stream is None else stream
+        binding.as_hybrid_attn_linear_state(self._h, self.workspace().data_ptr(), S.data_ptr(), z.data_ptr(),
+                                            st.cuda_stream)
+        return S, z
+
+    def last_status(self, stream=None) -> int:
+        import torch
+        st = torch.cuda.current_stream() if stream is None else stream
+        return binding.as_hybrid_attn_last_status(self._h, st.cuda_stream)
+
+    def close(self):
+        if getattr(self, "_h", None) is not None:
+            binding.as_hybrid_attn_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

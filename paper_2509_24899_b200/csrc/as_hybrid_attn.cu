@@ -1,0 +1,340 @@
+// Host side of libas_hybrid_attn: argument checking, the token split, workspace layout and
+// the launch sequence of the forward pass.  No arithmetic of the method runs here except the
+// integer token rule.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "as_internal.h"
+
+namespace {
+
+size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+// Token rule of section "Hybrid Attention" (T_S = { i : i mod R = 1 }, 1-indexed), applied to the
+// raster index inside each clipped spatial block; a block equal to the grid is the paper's rule.
+void build_token_split(const as_hybrid_attn_desc_t& d, std::vector<int32_t>& idx) {
+  idx.clear();
+  const int R = d.rate_den;
+  if (R == 0) return;
+  for (int t = 0; t < d.grid_t; ++t)
+    for (int h = 0; h < d.grid_h; ++h)
+      for (int w = 0; w < d.grid_w; ++w) {
+        const int n = (t * d.grid_h + h) * d.grid_w + w;
+        if (R == 1) { idx.push_back(n); continue; }
+        const int ot = t / d.blk_t * d.blk_t, oh = h / d.blk_h * d.blk_h, ow = w / d.blk_w * d.blk_w;
+        const int eh = std::min(d.blk_h, d.grid_h - oh), ew = std::min(d.blk_w, d.grid_w - ow);
+        const int l = ((t - ot) * eh + (h - oh)) * ew + (w - ow);
+        if (l % R == 0) idx.push_back(n);
+      }
+}
+
+as_status_t validate(const as_hybrid_attn_desc_t* d) {
+  if (!d) return AS_ERR_INVALID_ARG;
+  if (d->struct_size != sizeof(as_hybrid_attn_desc_t)) return AS_ERR_INVALID_ARG;
+  if (d->B <= 0 || d->H <= 0 || d->N <= 0) return AS_ERR_INVALID_ARG;
+  if (d->grid_t <= 0 || d->grid_h <= 0 || d->grid_w <= 0) return AS_ERR_INVALID_ARG;
+  if ((long long)d->grid_t * d->grid_h * d->grid_w != (long long)d->N) return AS_ERR_INVALID_ARG;
+  if (d->rate_den < 0) return AS_ERR_INVALID_ARG;
+  if (d->softmax_idx == nullptr && d->rate_den > 1 &&
+      (d->blk_t <= 0 || d->blk_h <= 0 || d->blk_w <= 0)) return AS_ERR_INVALID_ARG;
+  if (d->softmax_idx != nullptr) {
+    if (d->n_softmax < 0 || d->n_softmax > d->N) return AS_ERR_INVALID_ARG;
+    for (int i = 0; i < d->n_softmax; ++i) {
+      if (d->softmax_idx[i] < 0 || d->softmax_idx[i] >= d->N) return AS_ERR_INVALID_ARG;
+      if (i > 0 && d->softmax_idx[i] <= d->softmax_idx[i - 1]) return AS_ERR_INVALID_ARG;
+    }
+  }
+  if (d->stab_mode != AS_STAB_PAPER && d->stab_mode != AS_STAB_EXACT) return AS_ERR_INVALID_ARG;
+  if (d->kernel_path != AS_PATH_TENSOR && d->kernel_path != AS_PATH_SIMT) return AS_ERR_INVALID_ARG;
+  if (!(d->softmax_scale >= 0.f) || !std::isfinite(d->softmax_scale)) return AS_ERR_INVALID_ARG;
+  if (d->phi_dim <= 0 || d->poly_degree <= 0 || d->phi_layers <= 0) return AS_ERR_INVALID_ARG;
+  if (d->phi_dim % d->poly_degree != 0) return AS_ERR_INVALID_ARG;
+  // what this build has kernels for
+  if (d->d != 64 && d->d != 128) return AS_ERR_UNSUPPORTED;
+  if (d->phi_dim != d->d) return AS_ERR_UNSUPPORTED;
+  if (d->phi_layers != 1 || d->poly_degree > 2 || d->phi_act != AS_ACT_RELU) return AS_ERR_UNSUPPORTED;
+  if ((long long)d->B * d->H > 65535) return AS_ERR_UNSUPPORTED;
+  return AS_OK;
+}
+
+void layout_workspace(as_hybrid_attn_s* h) {
+  const auto& d = h->desc;
+  const size_t BH = (size_t)d.B * d.H;
+  as_ws_layout& w = h->ws;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
+  const bool compact = h->n_s > 0 && h->n_l > 0;      // at rate 1 the Q pass reads k, v directly
+  w.ks = take(compact ? BH * h->n_s * d.d * 2 : 0);
+  w.vs = take(compact ? BH * h->n_s * d.d * 2 : 0);
+  const bool lin = h->n_l > 0;
+  w.part_s = take(lin ? BH * h->n_chunks * d.phi_dim * d.d * 4 : 0);
+  w.part_z = take(lin ? BH * h->n_chunks * d.phi_dim * 4 : 0);
+  w.S = take(lin ? BH * d.phi_dim * d.d * 4 : 0);
+  w.z = take(lin ? BH * d.phi_dim * 4 : 0);
+  w.St = take(lin ? BH * d.phi_dim * d.d * 2 : 0);
+  w.total = std::max<size_t>(off, 256);
+  const size_t t = BH * d.N * d.d * 2;
+  off = w.total;
+  w.stage_q = take(t); w.stage_k = take(t); w.stage_v = take(t); w.stage_o = take(t);
+  w.total_host = off;
+}
+
+struct ProfileScope {
+  as_hybrid_attn_s* h; cudaStream_t st; int slot = -1;
+  ProfileScope(as_hybrid_attn_s* h_, cudaStream_t st_, int cls) : h(h_), st(st_) {
+    h->launches++;
+    if (h->profiling && h->ev_used < AS_MAX_PROFILE) {
+      slot = h->ev_used++;
+      h->ev_class[slot] = cls;
+      cudaEventRecord(h->ev[2 * slot], st);
+    }
+  }
+  ~ProfileScope() { if (slot >= 0) cudaEventRecord(h->ev[2 * slot + 1], st); }
+};
+
+}  // namespace
+
+extern "C" {
+
+const char* as_status_string(as_status_t s) {
+  switch (s) {
+    case AS_OK: return "ok";
+    case AS_ERR_INVALID_ARG: return "invalid argument";
+    case AS_ERR_UNSUPPORTED: return "unsupported configuration";
+    case AS_ERR_ARCH: return "device is not sm_100";
+    case AS_ERR_ALLOC: return "allocation failed";
+    case AS_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case AS_ERR_CUDA: return "CUDA call failed";
+    case AS_ERR_DEVICE_TIMEOUT: return "bounded wait inside a kernel expired";
+  }
+  return "unknown status";
+}
+
+as_status_t as_hybrid_attn_create(const as_hybrid_attn_desc_t* desc, as_hybrid_attn_t* out) {
+  if (!out) return AS_ERR_INVALID_ARG;
+  as_status_t vs = validate(desc);
+  if (vs != AS_OK) return vs;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+    cudaGetLastError(); return AS_ERR_CUDA;
+  }
+  if (major != 10) return AS_ERR_ARCH;
+
+  as_hybrid_attn_s* h = new (std::nothrow) as_hybrid_attn_s();
+  if (!h) return AS_ERR_ALLOC;
+  h->desc = *desc;
+  h->desc.softmax_idx = nullptr;                 // the caller's array is not kept
+  h->device = dev;
+  h->scale = desc->softmax_scale > 0.f ? desc->softmax_scale : 1.0f / std::sqrt((float)desc->d);
+  if (desc->softmax_idx) h->idx_host.assign(desc->softmax_idx, desc->softmax_idx + desc->n_softmax);
+  else build_token_split(*desc, h->idx_host);
+  h->n_s = (int)h->idx_host.size();
+  h->n_l = desc->N - h->n_s;
+  h->desc.n_softmax = h->n_s;
+
+  // K-pass split of the token axis: at most one CTA per SM over all (batch, head) pairs.
+  const int tiles = (desc->N + AS_TILE - 1) / AS_TILE;
+  int sms = 148;
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int BH = desc->B * desc->H;
+  int chunks = std::max(1, std::min(tiles, sms / BH));
+  h->chunk_tiles = (tiles + chunks - 1) / chunks;
+  h->n_chunks = (tiles + h->chunk_tiles - 1) / h->chunk_tiles;
+  layout_workspace(h);
+
+  std::vector<int32_t> rank(desc->N, -1);
+  for (int i = 0; i < h->n_s; ++i) rank[h->idx_host[i]] = i;
+  if (cudaMalloc(&h->d_sm_rank, sizeof(int32_t) * desc->N) != cudaSuccess ||
+      cudaMalloc(&h->d_status, 256) != cudaSuccess) {
+    cudaGetLastError(); as_hybrid_attn_destroy(h); return AS_ERR_ALLOC;
+  }
+  if (cudaMemcpy(h->d_sm_rank, rank.data(), sizeof(int32_t) * desc->N, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemset(h->d_status, 0, 256) != cudaSuccess) {
+    cudaGetLastError(); as_hybrid_attn_destroy(h); return AS_ERR_CUDA;
+  }
+  if (desc->kernel_path == AS_PATH_TENSOR && as_tensor_init() != cudaSuccess) {
+    cudaGetLastError(); as_hybrid_attn_destroy(h); return AS_ERR_CUDA;
+  }
+  *out = h;
+  return AS_OK;
+}
+
+as_status_t as_hybrid_attn_destroy(as_hybrid_attn_t h) {
+  if (!h) return AS_OK;
+  if (h->d_sm_rank) cudaFree(h->d_sm_rank);
+  if (h->d_status) cudaFree(h->d_status);
+  for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
+  delete h;
+  return AS_OK;
+}
+
+as_status_t as_hybrid_attn_workspace_bytes(as_hybrid_attn_t h, size_t* bytes) {
+  if (!h || !bytes) return AS_ERR_INVALID_ARG;
+  *bytes = h->ws.total;
+  return AS_OK;
+}
+
+as_status_t as_hybrid_attn_workspace_bytes_host(as_hybrid_attn_t h, size_t* bytes) {
+  if (!h || !bytes) return AS_ERR_INVALID_ARG;
+  *bytes = h->ws.total_host;
+  return AS_OK;
+}
+
+as_status_t as_hybrid_attn_softmax_tokens(as_hybrid_attn_t h, int32_t* count, int32_t* idx_host,
+                                          int32_t capacity) {
+  if (!h || !count) return AS_ERR_INVALID_ARG;
+  if (idx_host) {
+    if (capacity < h->n_s) return AS_ERR_INVALID_ARG;
+    std::memcpy(idx_host, h->idx_host.data(), sizeof(int32_t) * h->n_s);
+  }
+  *count = h->n_s;
+  return AS_OK;
+}
+
+as_status_t as_hybrid_attn_forward(as_hybrid_attn_t h, const void* q, const void* k, const void* v,
+                                   const as_phi_weights_t* w, void* out, float* aux,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!h || !q || !k || !v || !out) return AS_ERR_INVALID_ARG;
+  const auto& d = h->desc;
+  const bool lin = h->n_l > 0;
+  if (lin) {
+    if (!w || !w->wq1 || !w->wk1) return AS_ERR_INVALID_ARG;
+    if (w->bq1 || w->bk1 || w->wq2 || w->wk2 || w->bq2 || w->bk2) return AS_ERR_UNSUPPORTED;
+    if (((uintptr_t)w->wq1 | (uintptr_t)w->wk1) & 15) return AS_ERR_INVALID_ARG;
+  }
+  if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15) return AS_ERR_INVALID_ARG;
+  if (aux && ((uintptr_t)aux & 3)) return AS_ERR_INVALID_ARG;
+  if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < h->ws.total) return AS_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  char* ws = (char*)workspace;
+
+  as_launch_args a{};
+  a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;
+  a.wq = lin ? (const __nv_bfloat16*)w->wq1 : nullptr;
+  a.wk = lin ? (const __nv_bfloat16*)w->wk1 : nullptr;
+  a.out = (__nv_bfloat16*)out; a.aux = aux;
+  const bool compact = h->n_s > 0 && lin;
+  a.ks_w = compact ? (__nv_bfloat16*)(ws + h->ws.ks) : nullptr;
+  a.vs_w = compact ? (__nv_bfloat16*)(ws + h->ws.vs) : nullptr;
+  a.ks = compact ? a.ks_w : a.k;
+  a.vs = compact ? a.vs_w : a.v;
+  a.part_s = (float*)(ws + h->ws.part_s); a.part_z = (float*)(ws + h->ws.part_z);
+  a.S = (float*)(ws + h->ws.S); a.z = (float*)(ws + h->ws.z);
+  a.St = (__nv_bfloat16*)(ws + h->ws.St);
+  a.sm_rank = h->d_sm_rank; a.status = h->d_status;
+  a.B = d.B; a.H = d.H; a.N = d.N; a.d = d.d; a.F = d.phi_dim; a.P = d.poly_degree;
+  a.n_s = h->n_s; a.n_l = h->n_l; a.n_chunks = h->n_chunks; a.chunk_tiles = h->chunk_tiles;
+  a.scale = h->scale; a.stab_mode = d.stab_mode;
+
+  const bool simt = d.kernel_path == AS_PATH_SIMT;
+  cudaError_t e = cudaSuccess;
+  if (lin) {
+    { ProfileScope p(h, st, AS_KERNEL_KPASS);
+      e = simt ? as_simt_kpass(a, st) : as_tensor_kpass(a, st); }
+    if (e != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
+    { ProfileScope p(h, st, AS_KERNEL_REDUCE);
+      e = as_reduce_state(a, st); }
+    if (e != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
+  }
+  { ProfileScope p(h, st, AS_KERNEL_QPASS);
+    e = simt ? as_simt_qpass(a, st) : as_tensor_qpass(a, st); }
+  if (e != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
+  return AS_OK;
+}
+
+as_status_t as_hybrid_attn_forward_host(as_hybrid_attn_t h, const void* q_host, const void* k_host,
+                                        const void* v_host, const as_phi_weights_t* w,
+                                        void* out_host, void* workspace, size_t workspace_bytes,
+                                        void* cuda_stream) {
+  if (!h || !q_host || !k_host || !v_host || !out_host) return AS_ERR_INVALID_ARG;
+  if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < h->ws.total_host) return AS_ERR_WORKSPACE;
+  const auto& d = h->desc;
+  const size_t bytes = (size_t)d.B * d.H * d.N * d.d * 2;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  char* ws = (char*)workspace;
+  if (cudaMemcpyAsync(ws + h->ws.stage_q, q_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(ws + h->ws.stage_k, k_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(ws + h->ws.stage_v, v_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    cudaGetLastError(); return AS_ERR_CUDA;
+  }
+  as_status_t s = as_hybrid_attn_forward(h, ws + h->ws.stage_q, ws + h->ws.stage_k, ws + h->ws.stage_v, w,
+                                         ws + h->ws.stage_o, nullptr, workspace, h->ws.total, cuda_stream);
+  if (s != AS_OK) return s;
+  if (cudaMemcpyAsync(out_host, ws + h->ws.stage_o, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+    cudaGetLastError(); return AS_ERR_CUDA;
+  }
+  return AS_OK;
+}
+
+as_status_t as_hybrid_attn_linear_state(as_hybrid_attn_t h, const void* workspace, float* S_out,
+                                        float* z_out, void* cuda_stream) {
+  if (!h || !workspace) return AS_ERR_INVALID_ARG;
+  if (h->n_l == 0) return AS_ERR_INVALID_ARG;
+  const auto& d = h->desc;
+  const size_t BH = (size_t)d.B * d.H;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const char* ws = (const char*)workspace;
+  if (S_out && cudaMemcpyAsync(S_out, ws + h->ws.S, BH * d.phi_dim * d.d * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
+    cudaGetLastError(); return AS_ERR_CUDA;
+  }
+  if (z_out && cudaMemcpyAsync(z_out, ws + h->ws.z, BH * d.phi_dim * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
+    cudaGetLastError(); return AS_ERR_CUDA;
+  }
+  return AS_OK;
+}
+
+as_status_t as_hybrid_attn_last_status(as_hybrid_attn_t h, void* cuda_stream) {
+  if (!h) return AS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  uint32_t word = 0;
+  if (cudaStreamSynchronize(st) != cudaSuccess ||
+      cudaMemcpy(&word, h->d_status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError(); return AS_ERR_CUDA;
+  }
+  if (word != 0 && cudaMemset(h->d_status, 0, 4) != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
+  return (word & AS_DEV_TIMEOUT) ? AS_ERR_DEVICE_TIMEOUT : AS_OK;
+}
+
+as_status_t as_hybrid_attn_profile_enable(as_hybrid_attn_t h, int32_t enable) {
+  if (!h) return AS_ERR_INVALID_ARG;
+  if (enable && h->ev.empty()) {
+    h->ev.reserve(2 * AS_MAX_PROFILE);
+    for (int i = 0; i < 2 * AS_MAX_PROFILE; ++i) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
+      h->ev.push_back(e);
+    }
+    h->ev_class.assign(AS_MAX_PROFILE, 0);
+  }
+  h->profiling = enable != 0;
+  h->ev_used = 0;
+  return AS_OK;
+}
+
+as_status_t as_hybrid_attn_profile_read(as_hybrid_attn_t h, float* ms, int32_t* launches) {
+  if (!h || !ms || !launches) return AS_ERR_INVALID_ARG;
+  float acc[AS_NUM_KERNELS] = {0.f, 0.f, 0.f};
+  int32_t cnt[AS_NUM_KERNELS] = {0, 0, 0};
+  for (int i = 0; i < h->ev_used; ++i) {
+    if (cudaEventSynchronize(h->ev[2 * i + 1]) != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, h->ev[2 * i], h->ev[2 * i + 1]) != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
+    acc[h->ev_class[i]] += t;
+    cnt[h->ev_class[i]]++;
+  }
+  for (int c = 0; c < AS_NUM_KERNELS; ++c) { ms[c] = acc[c]; launches[c] = cnt[c]; }
+  h->ev_used = 0;
+  return AS_OK;
+}
+
+as_status_t as_hybrid_attn_launch_count(as_hybrid_attn_t h, uint64_t* count) {
+  if (!h || !count) return AS_ERR_INVALID_ARG;
+  *count = h->launches;
+  return AS_OK;
+}
+
+}  // extern "C"

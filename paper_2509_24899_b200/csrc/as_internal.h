@@ -1,0 +1,71 @@
+// Internal declarations shared by the translation units of libas_hybrid_attn.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "as_hybrid_attn.h"
+
+constexpr int AS_TILE = 128;            // tokens per tile in every kernel
+constexpr int AS_MAX_PROFILE = 1024;    // event pairs kept between two profile reads
+
+// Byte offsets of the workspace segments (all multiples of 256).
+struct as_ws_layout {
+  size_t ks = 0, vs = 0;                // compacted softmax K / V   [B*H, N_S, d] bf16
+  size_t part_s = 0, part_z = 0;        // per-chunk partial state   [B*H, chunks, F, d] / [.., F] fp32
+  size_t S = 0, z = 0;                  // final state               [B*H, F, d] / [B*H, F] fp32
+  size_t St = 0;                        // S transposed              [B*H, d, F] bf16 (MMA operand)
+  size_t total = 0;
+  size_t stage_q = 0, stage_k = 0, stage_v = 0, stage_o = 0, total_host = 0;
+};
+
+// Everything a kernel launch needs, resolved to device pointers.
+struct as_launch_args {
+  const __nv_bfloat16 *q, *k, *v, *wq, *wk;
+  __nv_bfloat16* out;
+  float* aux;
+  const __nv_bfloat16 *ks, *vs;         // softmax keys / values the Q pass reads (k, v themselves at R = 1)
+  __nv_bfloat16 *ks_w, *vs_w;           // where the K pass writes the compacted rows (NULL at R = 1)
+  float *part_s, *part_z, *S, *z;
+  __nv_bfloat16* St;
+  const int32_t* sm_rank;               // [N]: position in T_S, or -1 for a linear token
+  uint32_t* status;                     // device status word
+  int B, H, N, d, F, P;
+  int n_s, n_l;
+  int n_chunks, chunk_tiles;            // K-pass split of the token axis
+  float scale;
+  int stab_mode;
+};
+
+struct as_hybrid_attn_s {
+  as_hybrid_attn_desc_t desc;
+  int device = -1;
+  int n_s = 0, n_l = 0;
+  float scale = 0.f;
+  std::vector<int32_t> idx_host;        // sorted T_S
+  int32_t* d_sm_rank = nullptr;
+  uint32_t* d_status = nullptr;
+  int n_chunks = 1, chunk_tiles = 1;
+  as_ws_layout ws;
+  uint64_t launches = 0;
+  // profiling
+  bool profiling = false;
+  std::vector<cudaEvent_t> ev;          // 2 * AS_MAX_PROFILE events, created on first enable
+  std::vector<int> ev_class;
+  int ev_used = 0;
+};
+
+// Kernel launchers.  Each returns the launch's cudaError_t.
+cudaError_t as_simt_kpass(const as_launch_args& a, cudaStream_t st);
+cudaError_t as_simt_qpass(const as_launch_args& a, cudaStream_t st);
+cudaError_t as_reduce_state(const as_launch_args& a, cudaStream_t st);
+cudaError_t as_tensor_kpass(const as_launch_args& a, cudaStream_t st);
+cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st);
+// One-time set-up of the tensor path on the current device (driver entry points, smem opt-in).
+cudaError_t as_tensor_init();
+
+// Status bits written by kernels into as_launch_args::status.
+constexpr uint32_t AS_DEV_TIMEOUT = 1u;

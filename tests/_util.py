@@ -1,0 +1,106 @@
+"""Helpers shared by the GPU parity tests: input marshalling, oracle evaluation, error metrics.
+
+The expected values always come from `oracle/`; nothing computed on the GPU is fed to it.
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+from oracle import hybrid_attention as O
+from paper_2509_24899_b200 import workloads as W
+
+# Tolerances of the parity bar (bf16 inputs, fp32 accumulation).
+REL_L2_TOL = 5e-3
+MAX_ABS_TOL = 2e-2      # times the RMS of the oracle output
+
+
+def to_cuda_bf16(bits: np.ndarray):
+    import torch
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def from_cuda_bf16(t) -> np.ndarray:
+    import torch
+    return W.bf16_bits_to_f64(t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16))
+
+
+def oracle_inputs(data):
+    return {k: W.bf16_bits_to_f64(v) for k, v in data.items()}
+
+
+def errors(got: np.ndarray, ref: np.ndarray):
+    """(relative L2 error, max-abs error divided by the RMS of the reference)."""
+    diff = got - ref
+    rel_l2 = math.sqrt(float((diff ** 2).sum()) / max(float((ref ** 2).sum()), 1e-300))
+    rms = math.sqrt(float((ref ** 2).mean()))
+    return rel_l2, float(np.abs(diff).max()) / max(rms, 1e-300)
+
+
+def assert_parity(got, ref, what=""):
+    rel_l2, max_abs = errors(got, ref)
+    assert np.isfinite(got).all(), "%s: non-finite output" % what
+    assert rel_l2 <= REL_L2_TOL and max_abs <= MAX_ABS_TOL, \
+        "%s: rel-L2 %.3e (tol %.0e), max-abs/RMS %.3e (tol %.0e)" % (what, rel_l2, REL_L2_TOL, max_abs, MAX_ABS_TOL)
+    return rel_l2, max_abs
+
+
+def oracle_mask(wl):
+    return O.softmax_token_mask(wl.grid, wl.block, wl.rate)
+
+
+def balanced_gain(wl, stab_mode, sample_rows=48, seed=123):
+    """Gain g for W_q such that the median over sampled queries of lambda_i*den_L/den_S is 1.
+
+    With Glorot-random feature maps the linear branch outweighs the softmax branch by orders of
+    magnitude, and a wrong softmax branch would hide inside the tolerance.  Scaling W_q by g
+    (before bf16 rounding, as the generator does) makes both branches matter.  Uses the oracle only.
+    """
+    mask = oracle_mask(wl)
+    if mask.all() or not mask.any():
+        return 1.0
+    data = oracle_inputs(W.generate(wl, heads=1))
+    rng = np.random.default_rng(seed)
+    rows = np.sort(rng.choice(wl.N, size=min(sample_rows, wl.N), replace=False))
+    q, k, v = data["q"][0, 0], data["k"][0, 0], data["v"][0, 0]
+    _, z = O.linear_state(k, v, data["wk"][0], mask, wl.degree)
+    s = (q[rows] @ k[mask].T) / math.sqrt(wl.d)
+    c = s.max(1)
+    den_s = np.exp(s - c[:, None]).sum(1)
+    lam = np.exp(-c) if stab_mode == O.STAB_EXACT else np.ones_like(c)
+    wq32 = W.bf16_bits_to_f32(W.generate(wl, heads=1)["wq"][0])     # gain-1 weights (bf16 values)
+
+    def ratio(g):
+        wq = W.bf16_bits_to_f64(W.f32_to_bf16_bits(wq32 * np.float32(g)))
+        den_l = O.phi_features(q[rows], wq, wl.degree) @ z
+        return float(np.median(lam * den_l / den_s))
+
+    lo, hi = 1e-6, 1.0
+    if ratio(hi) <= 1.0:
+        return 1.0
+    for _ in range(60):
+        mid = math.sqrt(lo * hi)
+        if ratio(mid) > 1.0:
+            hi = mid
+        else:
+            lo = mid
+    return math.sqrt(lo * hi)
+
+
+def oracle_eval(wl, data64, stab_mode, rows=None):
+    """(y, aux) of the oracle for every head; `rows` selects query rows."""
+    return O.hybrid_attention(data64["q"], data64["k"], data64["v"], data64["wq"], data64["wk"],
+                              oracle_mask(wl), None, stab_mode, wl.degree, rows=rows)
+
+
+def oracle_state(wl, data64):
+    """S [B,H,F,d], z [B,H,F] of the oracle."""
+    mask = oracle_mask(wl)
+    B, H = data64["q"].shape[:2]
+    S = np.empty((B, H, wl.F, wl.d))
+    z = np.empty((B, H, wl.F))
+    for b in range(B):
+        for h in range(H):
+            S[b, h], z[b, h] = O.linear_state(data64["k"][b, h], data64["v"][b, h], data64["wk"][h], mask, wl.degree)
+    return S, z

@@ -1,0 +1,300 @@
+"""Parity of the CUDA library (through the C ABI) against the float64 oracle.
+
+Bar: relative L2 <= 5e-3 and max-abs <= 2e-2 x RMS(oracle output) for the bf16 output;
+bit-exact for the integer token split.  Small cases are compared element by element; the
+full-size configurations are compared on sampled query rows (every key still takes part in
+each sampled row) plus the complete linear state S, z.
+"""
+import dataclasses
+import math
+
+import numpy as np
+import pytest
+
+from oracle import hybrid_attention as O
+from paper_2509_24899_b200 import workloads as W
+from _util import (assert_parity, balanced_gain, errors, from_cuda_bf16, oracle_eval, oracle_inputs,
+                   oracle_mask, oracle_state, to_cuda_bf16)
+
+pytestmark = pytest.mark.gpu
+
+PATHS = ["simt"]
+FULL_PATH = "simt"          # path used at the full benchmark sizes
+MODES = [O.STAB_PAPER, O.STAB_EXACT]
+
+# ragged cases: N and N_S are not multiples of the 128-token tile
+SMALL = {
+    "ragged_d128": W.Workload("ragged_d128", B=1, H=2, d=128, F=128, grid=(3, 10, 13), block=(1, 6, 8),
+                              rate=4, seed=11),
+    "ragged_d64": W.Workload("ragged_d64", B=2, H=3, d=64, F=64, grid=(2, 9, 31), block=(1, 4, 4),
+                             rate=2, seed=12, rms_norm_qk=False),
+    "one_tile": W.Workload("one_tile", B=1, H=1, d=128, F=128, grid=(1, 5, 7), block=(1, 5, 7),
+                           rate=3, seed=13),
+    "paper_rule_1d": W.Workload("paper_rule_1d", B=1, H=2, d=128, F=128, grid=(1, 1, 1000),
+                                block=(1, 1, 1000), rate=8, seed=14),
+    "multi_chunk": W.Workload("multi_chunk", B=1, H=1, d=128, F=128, grid=(8, 30, 52), block=(1, 6, 8),
+                              rate=8, seed=15),
+}
+
+
+def _path(name):
+    from paper_2509_24899_b200 import AS_PATH_SIMT, AS_PATH_TENSOR
+    return {"simt": AS_PATH_SIMT, "tensor": AS_PATH_TENSOR}[name]
+
+
+def _run(wl, path, mode, gain=1.0, rows=None, heads=None, want_state=False, softmax_idx=None):
+    """Runs the library on wl's inputs; returns (gpu out, gpu aux, oracle y, oracle aux, extras)."""
+    import torch
+    from paper_2509_24899_b200 import HybridAttention
+    data = W.generate(wl, wq_gain=gain, heads=heads)
+    if heads is not None:
+        wl = dataclasses.replace(wl, H=heads)
+    dev = {k: to_cuda_bf16(v) for k, v in data.items()}
+    op = HybridAttention.from_workload(wl, stab_mode=mode, kernel_path=_path(path), softmax_idx=softmax_idx)
+    aux = torch.full((wl.B, wl.H, wl.N, 3), float("nan"), dtype=torch.float32, device="cuda")
+    out = op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], aux=aux)
+    torch.cuda.synchronize()
+    assert op.last_status() == 0
+    got = from_cuda_bf16(out)
+    got_aux = aux.cpu().numpy().astype(np.float64)
+    extras = {"op": op, "n_softmax": op.n_softmax, "indices": op.softmax_indices()}
+    if want_state and op.n_softmax < wl.N:
+        S, z = op.linear_state()
+        torch.cuda.synchronize()
+        extras["S"], extras["z"] = S.cpu().numpy().astype(np.float64), z.cpu().numpy().astype(np.float64)
+    d64 = oracle_inputs(data)
+    ref, ref_aux = oracle_eval(wl, d64, mode, rows=rows)
+    if rows is not None:
+        got, got_aux = got[:, :, rows], got_aux[:, :, rows]
+    extras["data64"] = d64
+    extras["wl"] = wl
+    return got, got_aux, ref, ref_aux, extras
+
+
+def _check_aux(got_aux, ref_aux, wl, n_softmax):
+    if n_softmax > 0:
+        np.testing.assert_allclose(got_aux[..., 0], ref_aux[..., 0], atol=2e-3, rtol=0)
+        assert errors(got_aux[..., 1], ref_aux[..., 1])[0] <= 5e-3
+    if n_softmax < wl.N:
+        assert errors(got_aux[..., 2], ref_aux[..., 2])[0] <= 5e-3
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("balanced", [False, True])
+def test_tiny_config(path, mode, balanced):
+    wl = W.CONFIGS["tiny"]
+    gain = balanced_gain(wl, mode) if balanced else 1.0
+    got, got_aux, ref, ref_aux, ex = _run(wl, path, mode, gain, want_state=True)
+    assert ex["n_softmax"] == 32
+    assert_parity(got, ref, "tiny/%s" % path)
+    _check_aux(got_aux, ref_aux, wl, 32)
+    S, z = oracle_state(wl, ex["data64"])
+    assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
+    if balanced:
+        lam = np.exp(-ref_aux[..., 0]) if mode == O.STAB_EXACT else 1.0
+        ratio = np.median(lam * ref_aux[..., 2] / ref_aux[..., 1])
+        assert 0.2 < ratio < 5.0          # both branches carry weight in this variant
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("name", sorted(SMALL))
+def test_small_ragged_cases(path, mode, name):
+    wl = SMALL[name]
+    gain = balanced_gain(wl, mode)
+    got, got_aux, ref, ref_aux, ex = _run(wl, path, mode, gain, want_state=True)
+    mask = oracle_mask(wl)
+    assert ex["indices"] == np.flatnonzero(mask).tolist()         # integer work: bit-exact
+    assert_parity(got, ref, "%s/%s" % (name, path))
+    _check_aux(got_aux, ref_aux, wl, int(mask.sum()))
+    S, z = oracle_state(wl, ex["data64"])
+    assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("rate", [0, 1])
+@pytest.mark.parametrize("name", ["ragged_d128", "ragged_d64"])
+def test_degenerate_rates(path, rate, name):
+    wl = SMALL[name].with_rate(rate)
+    got, got_aux, ref, ref_aux, ex = _run(wl, path, O.STAB_PAPER, want_state=(rate == 0))
+    assert ex["n_softmax"] == (wl.N if rate == 1 else 0)
+    ok = np.isfinite(ref).all(-1)          # rate 0: a query with all-zero features is NaN in both
+    assert ok.mean() > 0.99
+    assert_parity(got[ok], ref[ok], "%s/R%d/%s" % (name, rate, path))
+    _check_aux(got_aux[ok], ref_aux[ok], wl, ex["n_softmax"])
+    if rate == 1:
+        # rate 1 is plain softmax attention: cross-check with the library routine as well
+        import torch
+        d = ex["data64"]
+        sd = torch.nn.functional.scaled_dot_product_attention(
+            torch.from_numpy(d["q"]), torch.from_numpy(d["k"]), torch.from_numpy(d["v"])).numpy()
+        assert_parity(got, sd, "sdpa")
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_explicit_softmax_index_list(path):
+    wl = SMALL["ragged_d128"]
+    rng = np.random.default_rng(5)
+    idx = np.sort(rng.choice(wl.N, size=77, replace=False))
+    import torch
+    from paper_2509_24899_b200 import HybridAttention
+    data = W.generate(wl, wq_gain=2e-3)
+    dev = {k: to_cuda_bf16(v) for k, v in data.items()}
+    op = HybridAttention.from_workload(wl, kernel_path=_path(path), softmax_idx=idx.tolist())
+    out = op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"])
+    torch.cuda.synchronize()
+    assert op.softmax_indices() == idx.tolist()
+    d64 = oracle_inputs(data)
+    mask = np.zeros(wl.N, bool)
+    mask[idx] = True
+    ref, _ = O.hybrid_attention(d64["q"], d64["k"], d64["v"], d64["wq"], d64["wk"], mask)
+    assert_parity(from_cuda_bf16(out), ref, "explicit idx/%s" % path)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_key_permutation_within_sets_leaves_output_unchanged(path):
+    """Property that holds at any size: permuting keys inside T_S and inside T_L changes nothing."""
+    import torch
+    from paper_2509_24899_b200 import HybridAttention
+    wl = SMALL["ragged_d128"]
+    data = W.generate(wl, wq_gain=balanced_gain(wl, O.STAB_PAPER))
+    mask = oracle_mask(wl)
+    rng = np.random.default_rng(9)
+    perm = np.arange(wl.N)
+    for sel in (mask, ~mask):
+        ids = np.flatnonzero(sel)
+        perm[ids] = rng.permutation(ids)
+    dev = {k: to_cuda_bf16(v) for k, v in data.items()}
+    op = HybridAttention.from_workload(wl, kernel_path=_path(path))
+    a = from_cuda_bf16(op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"]))
+    kp = to_cuda_bf16(np.ascontiguousarray(data["k"][:, :, perm]))
+    vp = to_cuda_bf16(np.ascontiguousarray(data["v"][:, :, perm]))
+    b = from_cuda_bf16(op.forward(dev["q"], kp, vp, dev["wq"], dev["wk"]))
+    torch.cuda.synchronize()
+    assert errors(b, a)[0] <= 5e-3
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("balanced", [False, True])
+def test_wan17_full(path, mode, balanced):
+    wl = W.CONFIGS["wan17"]
+    gain = balanced_gain(wl, mode) if balanced else 1.0
+    got, got_aux, ref, ref_aux, ex = _run(wl, path, mode, gain, want_state=True)
+    assert ex["n_softmax"] == 975
+    assert_parity(got, ref, "wan17/%s" % path)
+    _check_aux(got_aux, ref_aux, wl, 975)
+    S, z = oracle_state(wl, ex["data64"])
+    assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
+
+
+def _sample_rows(N, n, seed):
+    rng = np.random.default_rng(seed)
+    rows = rng.choice(N, size=n - 4, replace=False)
+    return np.unique(np.concatenate([rows, [0, 1, N - 2, N - 1]]))      # include first / last tile rows
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("balanced", [False, True])
+def test_wan81_headline_sampled_rows(mode, balanced):
+    """Headline shape in the launch configuration the benchmark times (tensor path)."""
+    wl = W.CONFIGS["wan81"]
+    gain = balanced_gain(wl, mode) if balanced else 1.0
+    rows = _sample_rows(wl.N, 160, 1)
+    got, got_aux, ref, ref_aux, ex = _run(wl, FULL_PATH, mode, gain, rows=rows, want_state=True)
+    assert ex["n_softmax"] == 4095
+    assert ex["indices"] == np.flatnonzero(oracle_mask(wl)).tolist()
+    assert_parity(got, ref, "wan81")
+    _check_aux(got_aux, ref_aux, wl, 4095)
+    S, z = oracle_state(wl, ex["data64"])
+    assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
+
+
+@pytest.mark.parametrize("rate", [1, 4, 16, 0])
+def test_stack_layer_rates_sampled_rows(rate):
+    """One layer of each distinct rate of the 30-layer block-rate stack (rate 8 is the headline)."""
+    sched = W.stack_schedule(0)
+    layer = sched.index(rate)
+    wl = W.stack_layer(layer)
+    assert wl.rate == rate
+    gain = balanced_gain(wl, O.STAB_PAPER)
+    rows = _sample_rows(wl.N, 96, 2)
+    got, got_aux, ref, ref_aux, ex = _run(wl, FULL_PATH, O.STAB_PAPER, gain, rows=rows, heads=4,
+                                          want_state=(rate != 1))
+    assert ex["n_softmax"] == {1: 32760, 4: 8190, 16: 2100, 0: 0}[rate]
+    ok = np.isfinite(ref).all(-1)
+    assert ok.mean() > 0.99
+    assert_parity(got[ok], ref[ok], "stack R=%d" % rate)
+    _check_aux(got_aux[ok], ref_aux[ok], ex["wl"], ex["n_softmax"])
+    if rate != 1:
+        S, z = oracle_state(ex["wl"], ex["data64"])
+        assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
+
+
+def test_wan161_cfg_batch_sampled_rows():
+    wl = W.CONFIGS["wan161cfg"]
+    gain = balanced_gain(wl, O.STAB_PAPER)
+    rows = _sample_rows(wl.N, 64, 3)
+    got, got_aux, ref, ref_aux, ex = _run(wl, FULL_PATH, O.STAB_PAPER, gain, rows=rows)
+    assert ex["n_softmax"] == 4100
+    assert_parity(got, ref, "wan161cfg")
+    _check_aux(got_aux, ref_aux, wl, 4100)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_host_buffer_entry_point_matches_device_entry_point(path):
+    import torch
+    from paper_2509_24899_b200 import HybridAttention
+    wl = SMALL["ragged_d64"]
+    data = W.generate(wl, wq_gain=balanced_gain(wl, O.STAB_PAPER))
+    dev = {k: to_cuda_bf16(v) for k, v in data.items()}
+    op = HybridAttention.from_workload(wl, kernel_path=_path(path))
+    ref = op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"]).clone()
+    host = {k: torch.from_numpy(data[k].view(np.int16)).pin_memory() for k in ("q", "k", "v")}
+    out_host = torch.empty_like(host["q"]).pin_memory()
+    op.forward_host(host["q"], host["k"], host["v"], dev["wq"], dev["wk"], out_host)
+    torch.cuda.synchronize()
+    assert torch.equal(out_host, ref.view(torch.int16).cpu())
+
+
+def test_run_to_run_determinism_and_launch_count():
+    import torch
+    from paper_2509_24899_b200 import HybridAttention, binding
+    wl = SMALL["multi_chunk"]
+    data = W.generate(wl, wq_gain=1e-3)
+    dev = {k: to_cuda_bf16(v) for k, v in data.items()}
+    op = HybridAttention.from_workload(wl, kernel_path=_path(FULL_PATH))
+    a = op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"]).clone()
+    b = op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"]).clone()
+    torch.cuda.synchronize()
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    assert binding.as_hybrid_attn_launch_count(op.handle) == 6       # K pass, reduce, Q pass; twice
+    binding.as_hybrid_attn_profile_enable(op.handle, True)
+    op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"])
+    ms, cnt = binding.as_hybrid_attn_profile_read(op.handle)
+    assert cnt == [1, 1, 1] and all(t > 0 for t in ms)
+
+
+def test_gpu_argument_errors():
+    import torch
+    from paper_2509_24899_b200 import HybridAttention, binding, AsError
+    wl = SMALL["one_tile"]
+    op = HybridAttention.from_workload(wl)
+    data = {k: to_cuda_bf16(v) for k, v in W.generate(wl).items()}
+    out = torch.empty_like(data["q"])
+    ws = op.workspace()
+    with pytest.raises(AsError) as e:
+        binding.as_hybrid_attn_forward(op.handle, data["q"].data_ptr(), data["k"].data_ptr(), data["v"].data_ptr(),
+                                       data["wq"].data_ptr(), data["wk"].data_ptr(), out.data_ptr(), 0,
+                                       ws.data_ptr(), op.workspace_bytes - 1, 0)
+    assert e.value.status == binding.AS_ERR_WORKSPACE
+    with pytest.raises(AsError) as e:
+        binding.as_hybrid_attn_forward(op.handle, data["q"].data_ptr() + 2, data["k"].data_ptr(), data["v"].data_ptr(),
+                                       data["wq"].data_ptr(), data["wk"].data_ptr(), out.data_ptr(), 0,
+                                       ws.data_ptr(), op.workspace_bytes, 0)
+    assert e.value.status == binding.AS_ERR_INVALID_ARG
+    with pytest.raises(AsError) as e:      # linear tokens exist, so the feature-map weights are required
+        binding.as_hybrid_attn_forward(op.handle, data["q"].data_ptr(), data["k"].data_ptr(), data["v"].data_ptr(),
+                                       0, 0, out.data_ptr(), 0, ws.data_ptr(), op.workspace_bytes, 0)
+    assert e.value.status == binding.AS_ERR_INVALID_ARG
