@@ -246,6 +246,14 @@ def run_ours(args, wl):
     binding.as_hybrid_attn_profile_enable(op.handle, False)
     status = op.last_status()
 
+    if args.skip_extras:          # profiling runs: only the device-timed region
+        if rank == 0:
+            print(json.dumps({"ms_per_step": ms / args.steps, "kernel_ms": kms, "launches": int(launches),
+                              "device_status": status, "note": "--skip-extras: no e2e, no cpu baseline"}))
+        if world > 1:
+            dist.destroy_process_group()
+        return 0 if status == 0 else 1
+
     # end to end: host buffers in, host buffer out, copies inside the timed region
     host = {k: torch.from_numpy(data[k].view(np.int16)).pin_memory() for k in ("q", "k", "v")}
     out_host = torch.empty_like(host["q"]).pin_memory()
@@ -337,6 +345,8 @@ def main():
                     help="tiny | wan17 | wan81 | wan161cfg | stack:<layer>")
     ap.add_argument("--path", default="tensor", choices=["tensor", "simt"],
                     help="kernel path: tcgen05 tensor-core kernels (default) or the fp32 CUDA-core check path")
+    ap.add_argument("--skip-extras", action="store_true",
+                    help="only the device-timed steps (for profiler runs): no e2e, no CPU baseline")
     args = ap.parse_args()
     from paper_2509_24899_b200 import workloads as W
     if args.workload.startswith("stack:"):

