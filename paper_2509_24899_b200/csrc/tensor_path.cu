@@ -19,6 +19,7 @@
 
 #include "as_internal.h"
 #include "sm100_ptx.cuh"
+#include "sm100_tmem_wide.cuh"
 
 namespace {
 
@@ -245,60 +246,59 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       ok = mbar_wait_warp(bar(B_S + g), j & 1, wc);
       if (!ok) break;
       tc_fence_after();
-      const int valid = min(128, p.n_s - j * 128);    // keys of this tile that exist
-      // pass 1: row maximum of the tile
-      float mx = -INFINITY;
+      uint32_t sv[128];                               // this thread's row of the 128 x 128 score tile
+      tmem_ld128_sync(tSg, sv);
+      const int valid = p.n_s - j * 128;              // keys of this tile that exist (>= 128: all)
+      if (valid < 128) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        tmem_ld32(tSg + c * 32, x);
-        tmem_ld_wait(x);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float s = __uint_as_float(x[i]);
-          mx = (c * 32 + i < valid) ? fmaxf(mx, s) : mx;
-        }
+        for (int i = 0; i < 128; ++i) sv[i] = (i < valid) ? sv[i] : 0xff800000u;   // -inf: exp2 gives 0
       }
+      float mx0 = fmax3(__uint_as_float(sv[0]), __uint_as_float(sv[1]), __uint_as_float(sv[2]));
+      float mx1 = fmax3(__uint_as_float(sv[3]), __uint_as_float(sv[4]), __uint_as_float(sv[5]));
+#pragma unroll
+      for (int i = 6; i + 3 < 128; i += 4) {
+        mx0 = fmax3(mx0, __uint_as_float(sv[i]), __uint_as_float(sv[i + 1]));
+        mx1 = fmax3(mx1, __uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3]));
+      }
+      float mx = fmax3(mx0, mx1, fmaxf(__uint_as_float(sv[126]), __uint_as_float(sv[127])));
       mx *= p.scale_log2;
       m_true = fmaxf(m_true, mx);
-      if (j == 0) {
-        m_ref = mx;
-      } else {
-        const bool need = mx > m_ref + RESCALE_THRESHOLD;
-        if (__any_sync(0xffffffffu, need)) {
-          // O += P V of the previous tile has completed (its commit precedes this tile's S barrier)
-          const float f = need ? ex2(m_ref - mx) : 1.f;
-#pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            tmem_ld32(tOg + c * 32, x);
-            tmem_ld_wait(x);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) x[i] = __float_as_uint(__uint_as_float(x[i]) * f);
-            tmem_st32(tOg + c * 32, x);
-          }
-          tmem_st_wait();
-          l *= f;
-          if (need) m_ref = mx;
-        }
-      }
-      // pass 2: P = exp2(s * scale_log2 - m_ref) as bf16, written over the first 64 columns of S
-      float lsum = 0.f;
+      // The reference maximum only moves when the row maximum grew by more than 2^8; then O and l
+      // are rescaled (after P is out of the registers; the MMA that adds P V waits for this thread).
+      const bool need = (j > 0) && (mx > m_ref + RESCALE_THRESHOLD);
+      const float resc = need ? ex2(m_ref - mx) : 1.f;
+      if (j == 0 || need) m_ref = mx;
+      // P = exp2(s * scale_log2 - m_ref) as bf16, written over the first 64 columns of S
+      const float neg_m = -m_ref;
+      float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        tmem_ld32(tSg + c * 32, x);
-        tmem_ld_wait(x);
-        uint32_t w[16];
+        uint32_t pw[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float p0 = ex2(fmaf(__uint_as_float(x[2 * i]), p.scale_log2, -m_ref));
-          float p1 = ex2(fmaf(__uint_as_float(x[2 * i + 1]), p.scale_log2, -m_ref));
-          p0 = (c * 32 + 2 * i < valid) ? p0 : 0.f;
-          p1 = (c * 32 + 2 * i + 1 < valid) ? p1 : 0.f;
-          lsum += p0 + p1;
-          w[i] = pack_bf16(p0, p1);
+        for (int i = 0; i < 8; ++i) {
+          const int k = c * 32 + 4 * i;
+          const float p0 = ex2(fmaf(__uint_as_float(sv[k]), p.scale_log2, neg_m));
+          const float p1 = ex2(fmaf(__uint_as_float(sv[k + 1]), p.scale_log2, neg_m));
+          const float p2 = ex2(fmaf(__uint_as_float(sv[k + 2]), p.scale_log2, neg_m));
+          const float p3 = ex2(fmaf(__uint_as_float(sv[k + 3]), p.scale_log2, neg_m));
+          l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+          pw[2 * i] = pack_bf16(p0, p1);
+          pw[2 * i + 1] = pack_bf16(p2, p3);
         }
-        tmem_st16(tSg + c * 16, w);
+        tmem_st16(tSg + c * 16, pw);
       }
-      l += lsum;
+      l = l * resc + ((l0 + l1) + (l2 + l3));
+      if (__any_sync(0xffffffffu, need)) {
+        // O += P V of the previous tile has completed (its commit precedes this tile's S barrier)
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          tmem_ld32(tOg + c * 32, x);
+          tmem_ld_wait(x);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) x[i] = __float_as_uint(__uint_as_float(x[i]) * resc);
+          tmem_st32(tOg + c * 32, x);
+        }
+      }
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(bar(B_P + g));
