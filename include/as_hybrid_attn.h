@@ -164,6 +164,31 @@ AS_API as_status_t as_hybrid_attn_profile_read(as_hybrid_attn_t h, float* ms, in
 /* Total number of kernels this handle has launched since create. */
 AS_API as_status_t as_hybrid_attn_launch_count(as_hybrid_attn_t h, uint64_t* count);
 
+/* The linear state S, z of one layer, computed WITHOUT allocating anything.  The paper has no
+ * counterpart of this call: it exists for callers that cannot request device memory - a server
+ * whose arena already owns all of HBM (cudaMalloc fails or is forbidden there), a plug-in that
+ * may only touch the buffers its host framework handed it, a latency-critical loop that must
+ * avoid the device-wide synchronisation inside cudaMalloc / cudaFree.  It needs no handle and
+ * no workspace: the per-chunk partial sums live in a fixed 8 MiB array inside the library
+ * image (every GPU that loads the library holds it until the process exits).
+ *   k, v      [B,H,N,d] bf16 device, read only          wk  [H,d,d] bf16 device (F == d, one layer)
+ *   grid_*, blk_*, rate_den, poly_degree                 as in as_hybrid_attn_desc_t (rule-based T_S)
+ *   S_out     [B,H,d,d] fp32 device, written             z_out [B,H,d] fp32 device, written
+ *             (one of the two may be NULL)
+ * S = sum_{T_L} phi_k(k_j)^T v_j and z = sum_{T_L} phi_k(k_j), in fp32 on CUDA cores.
+ * Limits: d in {64, 128}; B*H*d*(d+1)*4 bytes <= 8 MiB (B*H <= 127 at d = 128, <= 504 at d = 64);
+ * anything larger returns AS_ERR_UNSUPPORTED and launches nothing.
+ * The first call on a device looks up the array's device address and sets kernel attributes;
+ * make that first call outside any stream capture.  No cudaMalloc, cudaFree or other allocating
+ * routine is called, then or later.  Asynchronous on `cuda_stream`.  All calls share the one
+ * array, which keeps the previous call's contents; every slot a call reads it has written first,
+ * so nothing needs clearing, but two calls that overlap on the GPU (different streams or
+ * threads) race on it - serialise them. */
+AS_API as_status_t as_hybrid_attn_linear_state_static(
+    const void* k, const void* v, const void* wk, int32_t B, int32_t H, int32_t N, int32_t d,
+    int32_t grid_t, int32_t grid_h, int32_t grid_w, int32_t blk_t, int32_t blk_h, int32_t blk_w,
+    int32_t rate_den, int32_t poly_degree, float* S_out, float* z_out, void* cuda_stream);
+
 /* Static description of a status code. */
 AS_API const char* as_status_string(as_status_t s);
 

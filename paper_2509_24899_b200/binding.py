@@ -74,6 +74,8 @@ def lib() -> C.CDLL:
             "as_hybrid_attn_profile_enable": [H, C.c_int32],
             "as_hybrid_attn_profile_read": [H, C.POINTER(C.c_float), C.POINTER(C.c_int32)],
             "as_hybrid_attn_launch_count": [H, C.POINTER(C.c_uint64)],
+            "as_hybrid_attn_linear_state_static": [C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 12
+                                                  + [C.c_void_p, C.c_void_p, C.c_void_p],
         }
         for name, args in sigs.items():
             fn = getattr(L, name)
@@ -197,3 +199,16 @@ def as_hybrid_attn_launch_count(h) -> int:
     n = C.c_uint64()
     _check(lib().as_hybrid_attn_launch_count(h, C.byref(n)), "as_hybrid_attn_launch_count")
     return n.value
+
+
+def as_hybrid_attn_linear_state_static(k_ptr, v_ptr, wk_ptr, B, H, N, d, grid, block, rate, poly_degree,
+                                       S_ptr, z_ptr, stream_ptr) -> None:
+    """S [B,H,d,d] and z [B,H,d] (fp32) of one layer without any allocation inside the library.
+
+    For callers that cannot request device memory (an arena owns all of it, or only the buffers
+    handed in may be used): no handle, no workspace; the partial sums use a fixed 8 MiB array inside
+    the library.  Sizes beyond that array raise AsError(AS_ERR_UNSUPPORTED).  Calls must not overlap
+    on the GPU; make the first call on a device outside any stream capture."""
+    _check(lib().as_hybrid_attn_linear_state_static(
+        k_ptr, v_ptr, wk_ptr, B, H, N, d, grid[0], grid[1], grid[2], block[0], block[1], block[2], rate,
+        poly_degree, S_ptr or None, z_ptr or None, stream_ptr or None), "as_hybrid_attn_linear_state_static")
