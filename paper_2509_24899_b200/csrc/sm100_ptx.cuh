@@ -42,21 +42,25 @@ AS_DEV bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait.  Gives up after `limit_ns`, or as soon as another thread of the CTA has given up;
-// then it raises the CTA's abort flag and the global status bit and returns false.
+// Bounded wait.  Gives up after about `kWaitLimitCycles` SM clocks (roughly a second), or as soon as
+// another thread of the CTA has given up; then it raises the CTA's abort flag and the global status bit
+// and returns false.  The clock is only looked at every 64 failed polls, so a wait that is satisfied
+// quickly costs nothing beyond the polls themselves.
 struct WaitCtx {
   uint32_t* status;             // global status word
   volatile uint32_t* abort;     // shared-memory flag of this CTA
 };
-constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;   // 1 s
+constexpr long long kWaitLimitCycles = 2000ll * 1000ll * 1000ll;
 
 AS_DEV bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w) {
   if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = globaltimer_ns();
+  long long t0 = 0;
   uint32_t it = 0;
   while (!mbar_try_wait(bar, parity)) {
-    if ((++it & 31u) == 0u) {
-      if (*w.abort != 0u || globaltimer_ns() - t0 > kWaitLimitNs) {
+    if ((++it & 63u) == 0u) {
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      if (*w.abort != 0u || now - t0 > kWaitLimitCycles) {
         *w.abort = 1u;
         atomicOr(w.status, 1u);
         return false;

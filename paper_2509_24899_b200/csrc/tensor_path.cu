@@ -59,23 +59,25 @@ AS_DEV void load_tile(uint32_t dst, const CUtensorMap* m, uint32_t bar, int y0, 
   for (int b = 0; b < D / 64; ++b) tma_load_3d(dst + b * BOX_BYTES, m, bar, b * 64, y0, z);
 }
 
+// Shared-memory descriptors are built once per tile; the k-steps of one MMA chain only add a byte
+// offset (in 16-byte units) to the address field, which keeps the issuing thread's instruction count low.
+AS_DEV uint64_t kmajor_desc(uint32_t smem) { return make_sdesc(smem, 16, 1024); }        // [rows x 64] boxes, K-major
+AS_DEV uint64_t mnmajor_desc(uint32_t smem) { return make_sdesc(smem, BOX_BYTES, 1024); } // k-rows x [64-column boxes], MN-major
+
 // D[tmem] (+)= A[smem, K-major, 128 x KD] * B[smem, K-major, NB x KD]^T
 template <int KD>
-AS_DEV void issue_kmajor(uint32_t d_tmem, uint32_t a_smem, uint32_t b_smem, uint32_t idesc, bool acc) {
+AS_DEV void issue_kmajor(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool acc) {
 #pragma unroll
   for (int kk = 0; kk < KD / 16; ++kk) {
-    const uint32_t off = (kk / 4) * BOX_BYTES + (kk % 4) * 32;
-    mma_ss(d_tmem, make_sdesc(a_smem + off, 16, 1024), make_sdesc(b_smem + off, 16, 1024), idesc,
-           (acc || kk > 0) ? 1u : 0u);
+    const uint64_t off = (uint64_t)(((kk / 4) * BOX_BYTES + (kk % 4) * 32) >> 4);
+    mma_ss(d_tmem, a_desc + off, b_desc + off, idesc, (acc || kk > 0) ? 1u : 0u);
   }
 }
 // D[tmem] (+)= A[tmem, 128 lanes x 128 k as packed bf16] * B[smem, MN-major: 128 k-rows x NB cols]
-AS_DEV void issue_tmemA_mnB(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_smem, uint32_t idesc, bool acc) {
+AS_DEV void issue_tmemA_mnB(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool acc) {
 #pragma unroll
-  for (int kk = 0; kk < 8; ++kk) {
-    mma_ts(d_tmem, a_tmem + kk * 8, make_sdesc(b_smem + kk * 2048, BOX_BYTES, 1024), idesc,
-           (acc || kk > 0) ? 1u : 0u);
-  }
+  for (int kk = 0; kk < 8; ++kk)
+    mma_ts(d_tmem, a_tmem + kk * 8, b_desc + (uint64_t)((kk * 2048) >> 4), idesc, (acc || kk > 0) ? 1u : 0u);
 }
 
 // Writes 32 consecutive columns [c0, c0+32) of row `row` of a swizzled [128 x D] bf16 tile.
@@ -179,22 +181,40 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       if (ok) {
         tc_fence_after();
         if (lane == 0) {
-          for (int g = 0; g < 2; ++g) { issue_kmajor<D>(tS[g], sQ[g], sKV(0), ID_QK, false); tc_commit(bar(B_S + g)); }
+          for (int g = 0; g < 2; ++g) { issue_kmajor<D>(tS[g], kmajor_desc(sQ[g]), kmajor_desc(sKV(0)), ID_QK, false); tc_commit(bar(B_S + g)); }
           tc_commit(bar(B_EMPTY + 0));
         }
         __syncwarp();
       }
       for (int j = 0; ok && j < nkv; ++j) {
-        for (int g = 0; ok && g < 2; ++g) {
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+          if (!ok) break;
+          // operands of the whole block are prepared before the wait, so that the issue itself is short
+          uint64_t dv[8], dq[8], dk[8];
+          uint32_t ap[8];
+          {
+            const uint64_t v0 = mnmajor_desc(sKV(2 * j + 1)), q0 = kmajor_desc(sQ[g]), k0 = kmajor_desc(sKV(2 * j + 2));
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+              const uint64_t off = (uint64_t)(((kk / 4) * BOX_BYTES + (kk % 4) * 32) >> 4);
+              dv[kk] = v0 + (uint64_t)((kk * 2048) >> 4);
+              dq[kk] = q0 + off;
+              dk[kk] = k0 + off;
+              ap[kk] = tS[g] + kk * 8;
+            }
+          }
           ok = mbar_wait_warp(bar(B_P + g), j & 1, wc);
           if (ok && g == 0) ok = full_wait(2 * j + 1);
           if (ok && g == 0 && j + 1 < nkv) ok = full_wait(2 * j + 2);
           if (!ok) break;
           tc_fence_after();
           if (lane == 0) {
-            issue_tmemA_mnB(tO[g], tS[g], sKV(2 * j + 1), ID_PV, j > 0);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) mma_ts(tO[g], ap[kk], dv[kk], ID_PV, (j > 0 || kk > 0) ? 1u : 0u);
             if (j + 1 < nkv) {
-              issue_kmajor<D>(tS[g], sQ[g], sKV(2 * j + 2), ID_QK, false);
+#pragma unroll
+              for (int kk = 0; kk < D / 16; ++kk) mma_ss(tS[g], dq[kk], dk[kk], ID_QK, kk > 0 ? 1u : 0u);
               tc_commit(bar(B_S + g));
             } else if (!p.lin) {
               tc_commit(bar(B_O + g));
@@ -214,7 +234,7 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       if (ok) {
         tc_fence_after();
         if (lane == 0) {
-          for (int g = 0; g < 2; ++g) { issue_kmajor<D>(tS[g], sQ[g], sKV(2 * nkv), ID_PHI, false); tc_commit(bar(B_S + g)); }
+          for (int g = 0; g < 2; ++g) { issue_kmajor<D>(tS[g], kmajor_desc(sQ[g]), kmajor_desc(sKV(2 * nkv)), ID_PHI, false); tc_commit(bar(B_S + g)); }
         }
         __syncwarp();
         ok = full_wait(2 * nkv + 1);
@@ -224,7 +244,7 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         if (!ok) break;
         tc_fence_after();
         if (lane == 0) {
-          issue_kmajor<F>(tO[g], sQ[g], sKV(2 * nkv + 1), ID_LIN, nkv > 0);
+          issue_kmajor<F>(tO[g], kmajor_desc(sQ[g]), kmajor_desc(sKV(2 * nkv + 1)), ID_LIN, nkv > 0);
           tc_commit(bar(B_O + g));
         }
         __syncwarp();
@@ -270,24 +290,26 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       if (j == 0 || need) m_ref = mx;
       // P = exp2(s * scale_log2 - m_ref) as bf16, written over the first 64 columns of S
       const float neg_m = -m_ref;
-      float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+      // packed fp32x2 arithmetic halves the instruction count of the scaling and of the row sum
+      const float2 scale2 = make_float2(p.scale_log2, p.scale_log2), negm2 = make_float2(neg_m, neg_m);
+      float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t pw[16];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int k = c * 32 + 4 * i;
-          const float p0 = ex2(fmaf(__uint_as_float(sv[k]), p.scale_log2, neg_m));
-          const float p1 = ex2(fmaf(__uint_as_float(sv[k + 1]), p.scale_log2, neg_m));
-          const float p2 = ex2(fmaf(__uint_as_float(sv[k + 2]), p.scale_log2, neg_m));
-          const float p3 = ex2(fmaf(__uint_as_float(sv[k + 3]), p.scale_log2, neg_m));
-          l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-          pw[2 * i] = pack_bf16(p0, p1);
-          pw[2 * i + 1] = pack_bf16(p2, p3);
+          const float2 xa = __ffma2_rn(make_float2(__uint_as_float(sv[k]), __uint_as_float(sv[k + 1])), scale2, negm2);
+          const float2 xb = __ffma2_rn(make_float2(__uint_as_float(sv[k + 2]), __uint_as_float(sv[k + 3])), scale2, negm2);
+          const float2 pa = make_float2(ex2(xa.x), ex2(xa.y)), pb = make_float2(ex2(xb.x), ex2(xb.y));
+          la = __fadd2_rn(la, pa);
+          lb = __fadd2_rn(lb, pb);
+          pw[2 * i] = pack_bf16(pa.x, pa.y);
+          pw[2 * i + 1] = pack_bf16(pb.x, pb.y);
         }
         tmem_st16(tSg + c * 16, pw);
       }
-      l = l * resc + ((l0 + l1) + (l2 + l3));
+      l = l * resc + ((la.x + la.y) + (lb.x + lb.y));
       if (__any_sync(0xffffffffu, need)) {
         // O += P V of the previous tile has completed (its commit precedes this tile's S barrier)
 #pragma unroll
@@ -484,7 +506,7 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         if (!ok) break;
         tc_fence_after();
         if (lane == 0) {
-          issue_kmajor<D>(tD1[t & 1], sW, sK(st), ID_PHI, false);
+          issue_kmajor<D>(tD1[t & 1], kmajor_desc(sW), kmajor_desc(sK(st)), ID_PHI, false);
           tc_commit(bar(B_D1 + (t & 1)));
         }
         __syncwarp();
@@ -495,7 +517,7 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         if (!ok) break;
         tc_fence_after();
         if (lane == 0) {
-          issue_tmemA_mnB(tAcc, tD1[u & 1], sV(st), ID_ACC, u > 0);
+          issue_tmemA_mnB(tAcc, tD1[u & 1], mnmajor_desc(sV(st)), ID_ACC, u > 0);
           tc_commit(bar(B_EMPTY + st));
           if (u == nt - 1) tc_commit(bar(B_DONE));
         }
