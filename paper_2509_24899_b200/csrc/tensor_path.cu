@@ -594,10 +594,11 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         for (int i = 0; i < 16; ++i) {
           float a0 = fmaxf(__uint_as_float(x[2 * i]), 0.f), a1 = fmaxf(__uint_as_float(x[2 * i + 1]), 0.f);
           if (squared) { a0 *= a0; a1 *= a1; }
-          a0 = ((mask >> (2 * i)) & 1u) ? bf16_round(a0) : 0.f;
-          a1 = ((mask >> (2 * i + 1)) & 1u) ? bf16_round(a1) : 0.f;
-          zacc += a0 + a1;
+          a0 = ((mask >> (2 * i)) & 1u) ? a0 : 0.f;
+          a1 = ((mask >> (2 * i + 1)) & 1u) ? a1 : 0.f;
           w[i] = pack_bf16(a0, a1);
+          // z sums the features as the MMA sees them: the bf16 values, read back out of the packed word
+          zacc += __uint_as_float(w[i] << 16) + __uint_as_float(w[i] & 0xffff0000u);
         }
         tmem_st16(tD1[b] + lane_off + c * 16, w);
       }
