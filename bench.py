@@ -335,6 +335,46 @@ def run_ours(args, wl):
     return rc
 
 
+def run_stack(args):
+    """The 30-layer block-rate stack: one timed layer per distinct rate, per-layer and summed time against
+    all layers running full softmax (rate 1).  Prints one JSON line of its own; not the headline line."""
+    import numpy as np
+    import torch
+    from paper_2509_24899_b200 import HybridAttention, workloads as W
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; the product path has no CPU fallback")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    sched = W.stack_schedule(0)
+    per_rate = {}
+    stream = torch.cuda.current_stream()
+    for rate in W.STACK_RATES:
+        wl = W.stack_layer(sched.index(rate))
+        data = W.generate(wl)
+        dev = {k: torch.from_numpy(v.view(np.int16)).cuda().view(torch.bfloat16) for k, v in data.items()}
+        op = HybridAttention.from_workload(wl)
+        out = torch.empty_like(dev["q"])
+        steps = max(3, args.steps // (10 if rate == 1 else 1))
+        for _ in range(3):
+            op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], out=out, stream=stream)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], out=out, stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        assert op.last_status() == 0
+        per_rate[rate] = {"ms_per_layer": e0.elapsed_time(e1) / steps, "layers": sched.count(rate),
+                          "n_softmax": op.n_softmax, "steps": steps}
+        del op, dev, out
+    total = sum(v["ms_per_layer"] * v["layers"] for v in per_rate.values())
+    all_softmax = per_rate[1]["ms_per_layer"] * len(sched)
+    print(json.dumps({"workload": "stack", "schedule": sched, "per_rate": {str(k): v for k, v in per_rate.items()},
+                      "stack_ms": total, "all_softmax_ms": all_softmax, "speedup_vs_all_softmax": all_softmax / total,
+                      "dtype": "bf16", "data": "synthetic"}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -342,13 +382,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="wan81",
-                    help="tiny | wan17 | wan81 | wan161cfg | stack:<layer>")
+                    help="tiny | wan17 | wan81 | wan161cfg | stack:<layer> | stack (all five rates, summed)")
     ap.add_argument("--path", default="tensor", choices=["tensor", "simt"],
                     help="kernel path: tcgen05 tensor-core kernels (default) or the fp32 CUDA-core check path")
     ap.add_argument("--skip-extras", action="store_true",
                     help="only the device-timed steps (for profiler runs): no e2e, no CPU baseline")
     args = ap.parse_args()
     from paper_2509_24899_b200 import workloads as W
+    if args.workload == "stack":
+        return run_stack(args)
     if args.workload.startswith("stack:"):
         wl = W.stack_layer(int(args.workload.split(":")[1]))
     else:
