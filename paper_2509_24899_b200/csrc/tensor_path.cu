@@ -414,7 +414,7 @@ struct KParams {
 };
 
 constexpr int K_THREADS = 256;           // warps 0-3: feature warps; 4: TMA; 5: MMA; 6-7: gather
-constexpr int K_STAGES = 2;
+constexpr int K_STAGES = 3;
 
 template <int D>
 struct KLayout {
@@ -527,18 +527,23 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   } else if (warp >= 6) {
     // ------------------------------------------------------------ gather of softmax-token rows
     const int gw = warp - 6;
+    // rows handled by this warp: gw*64 .. gw*64+63; two ranks per lane.  The ranks of tile t + 1 are
+    // fetched while tile t is being copied, so that the global-load latency stays off the critical path.
+    auto load_ranks = [&](int t, int (&rk)[2]) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int n = (t_begin + t) * 128 + gw * 64 + e * 32 + lane;
+        rk[e] = (t < nt && n < p.N && p.ks_w != nullptr) ? p.sm_rank[n] : -1;
+      }
+    };
+    int rk_next[2];
+    load_ranks(0, rk_next);
     for (int t = 0; t < nt; ++t) {
       const int st = t % K_STAGES;
+      int rk[2] = {rk_next[0], rk_next[1]};
+      load_ranks(t + 1, rk_next);
       if (!mbar_wait_warp(bar(B_FULL + st), (t / K_STAGES) & 1, wc)) break;
       if (p.ks_w != nullptr) {
-        const int n0 = (t_begin + t) * 128;
-        // rows handled by this warp: gw*64 .. gw*64+63; two ranks per lane
-        int rk[2];
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const int n = n0 + gw * 64 + e * 32 + lane;
-          rk[e] = (n < p.N) ? p.sm_rank[n] : -1;
-        }
         const uint8_t* kt = smem + L::KV_OFF + st * 2 * L::TILE;
         const uint8_t* vt = kt + L::TILE;
         constexpr int CH = D / 8;                          // 16-byte chunks per row
@@ -571,14 +576,19 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     float zacc = 0.f;
     bool ok = true;
     uint32_t x[32];
+    // which of a tile's 128 tokens are linear tokens (inside the sequence, not softmax tokens); the table
+    // entry of tile t + 1 is fetched while tile t is processed
+    auto is_linear = [&](int t) {
+      const int n = (t_begin + t) * 128 + f;
+      return (t < nt) && (n < p.N) && (p.sm_rank[n] < 0);
+    };
+    bool lin_next = is_linear(0);
     for (int t = 0; t < nt; ++t) {
       const int b = t & 1;
-      // which of the tile's 128 tokens are linear tokens (inside the sequence, not softmax tokens)
       {
-        const int n = (t_begin + t) * 128 + f;
-        const bool lin_tok = (n < p.N) && (p.sm_rank[n] < 0);
-        const uint32_t bits = __ballot_sync(0xffffffffu, lin_tok);
+        const uint32_t bits = __ballot_sync(0xffffffffu, lin_next);
         if (lane == 0) sMask[b * 4 + warp] = bits;
+        lin_next = is_linear(t + 1);
       }
       named_barrier_sync(1, 128);
       ok = mbar_wait_warp(bar(B_D1 + b), (t >> 1) & 1, wc);
