@@ -56,6 +56,27 @@ def bytes_per_layer(wl):
     return 4 * wl.B * wl.H * wl.N * wl.d * 2
 
 
+def rank_workload(wl, rank):
+    """Every rank draws its own layer input (independent batches: weak scaling, no exchange step)."""
+    import dataclasses
+    return dataclasses.replace(wl, seed=wl.seed + rank)
+
+
+def max_over_ranks(values, device):
+    """Element-wise maximum of a list of per-rank numbers over all ranks (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_value(wl, world, steps, ms):
+    """Tokens per second of the whole job: every rank processed `steps` layers of B*N tokens in `ms`."""
+    return wl.B * wl.N * world * steps / (ms * 1e-3)
+
+
 class ClockSampler:
     """Samples SM clock and clock-event reasons of one GPU through NVML in a background thread."""
 
@@ -214,7 +235,7 @@ def run_ours(args, wl):
         torch.cuda.synchronize()
 
     # every rank draws its own layer input (independent batches: weak scaling, no exchange step)
-    wl_r = dataclasses.replace(wl, seed=wl.seed + rank)
+    wl_r = rank_workload(wl, rank)
     data = W.generate(wl_r)
     to_dev = lambda b: torch.from_numpy(b.view(np.int16)).cuda().view(torch.bfloat16)
     dev = {k: to_dev(v) for k, v in data.items()}
@@ -269,13 +290,9 @@ def run_ours(args, wl):
     e2e_ms = e0.elapsed_time(e1)
     sampler.stop()
 
-    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, e2e_ms = t.tolist()
-    tokens = wl.B * wl.N * world
-    value = tokens * args.steps / (ms * 1e-3)
-    e2e_value = tokens * e2e_steps / (e2e_ms * 1e-3)
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms], "cuda")
+    value = whole_job_value(wl, world, args.steps, ms)
+    e2e_value = whole_job_value(wl, world, e2e_steps, e2e_ms)
 
     rc = 0
     if rank == 0:
