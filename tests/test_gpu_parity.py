@@ -153,6 +153,35 @@ def test_explicit_softmax_index_list(path):
 
 
 @pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("mode", MODES)
+def test_late_dominant_keys_move_the_reference_maximum(path, mode):
+    """Softmax keys late in the sequence are scaled up so that the row maximum grows by far more than 2^8
+    after the first key tiles: the kernels have to rescale their running sums on the way."""
+    import torch
+    from paper_2509_24899_b200 import HybridAttention
+    wl = SMALL["multi_chunk"]                       # N = 12480, 1560 softmax tokens = 13 key tiles
+    data = W.generate(wl, wq_gain=balanced_gain(wl, mode))
+    mask = oracle_mask(wl)
+    idx = np.flatnonzero(mask)
+    k32 = W.bf16_bits_to_f32(data["k"]).copy()
+    k32[:, :, idx[700:703]] *= 6.0                  # tile 5: scores up to ~6x the usual maximum
+    k32[:, :, idx[1500:1502]] *= 12.0               # last tile: larger again
+    data["k"] = W.f32_to_bf16_bits(k32)
+    dev = {k: to_cuda_bf16(v) for k, v in data.items()}
+    op = HybridAttention.from_workload(wl, stab_mode=mode, kernel_path=_path(path))
+    aux = torch.full((wl.B, wl.H, wl.N, 3), float("nan"), dtype=torch.float32, device="cuda")
+    out = op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], aux=aux)
+    torch.cuda.synchronize()
+    assert op.last_status() == 0
+    d64 = oracle_inputs(data)
+    rows = _sample_rows(wl.N, 512, 7)
+    ref, ref_aux = oracle_eval(wl, d64, mode, rows=rows)
+    assert (ref_aux[..., 0] > 12.0).mean() > 0.2   # the scaled keys do dominate many rows (c_i far above the usual ~4)
+    assert_parity(from_cuda_bf16(out)[:, :, rows], ref, "late dominant keys/%s" % path, strict=False)
+    _check_aux(aux.cpu().numpy().astype(np.float64)[:, :, rows], ref_aux, wl, int(mask.sum()))
+
+
+@pytest.mark.parametrize("path", PATHS)
 def test_key_permutation_within_sets_leaves_output_unchanged(path):
     """Property that holds at any size: permuting keys inside T_S and inside T_L changes nothing."""
     import torch
