@@ -83,7 +83,7 @@ typedef struct {
                                       NULL selects the rule above                                   */
   int32_t  n_softmax;              /* length of softmax_idx (ignored when it is NULL)              */
   int32_t  phi_dim;                /* F: output width of the feature map, in {64, 128}, == P * D'   */
-  int32_t  phi_layers;             /* embedding-network depth; 1 is supported                       */
+  int32_t  phi_layers;             /* embedding-network depth: 1, or 2 (tensor path, phi_hidden == d) */
   int32_t  phi_hidden;             /* hidden width when phi_layers == 2 (unused otherwise)          */
   int32_t  poly_degree;            /* P: part p (1-based) of the activation is raised to power p;
                                       1 or 2 is supported                                            */
@@ -94,8 +94,11 @@ typedef struct {
 } as_hybrid_attn_desc_t;
 
 /* Feature-map weights, DEVICE pointers, bf16, row-major with the output feature as the slow
- * index: w*1 is [H, F, d] when phi_layers == 1.  Biases and second layers must be NULL in this
- * build.  phi(x) = [a_1, a_2^2] with a = ReLU(W x) split into P contiguous parts. */
+ * index ("Characterization of phi": an embedding network, then the polynomial parts).
+ *   phi_layers == 1:  w*1 is [H, F, d];                        a = ReLU(W_1 x)
+ *   phi_layers == 2:  w*1 is [H, hidden, d], w*2 is [H, F, hidden];  a = ReLU(W_2 ReLU(W_1 x))
+ * phi(x) = [a_1, a_2^2]: a split into P contiguous parts, part p to the power p.  Biases must be
+ * NULL in this build; w*2 must be NULL when phi_layers == 1. */
 typedef struct {
   const void *wq1, *bq1, *wq2, *bq2;
   const void *wk1, *bk1, *wk2, *bk2;

@@ -15,11 +15,12 @@ __all__ = ["binding", "HybridAttention", "AS_PATH_SIMT", "AS_PATH_TENSOR", "AS_S
 class HybridAttention:
     """One layer geometry bound to the current CUDA device.
 
-    q, k, v: torch.bfloat16 CUDA tensors [B, H, N, d]; wq, wk: bfloat16 [H, F, d].
+    q, k, v: torch.bfloat16 CUDA tensors [B, H, N, d]; wq, wk: bfloat16 [H, F, d]; with phi_layers=2 the
+    feature map is relu(relu(x wq^T) wq2^T) before the powers, wq2, wk2: bfloat16 [H, F, F].
     """
 
     def __init__(self, B, H, N, d, grid, block, rate, phi_dim=None, poly_degree=2, softmax_scale=0.0,
-                 stab_mode=AS_STAB_PAPER, kernel_path=AS_PATH_TENSOR, softmax_idx=None):
+                 stab_mode=AS_STAB_PAPER, kernel_path=AS_PATH_TENSOR, softmax_idx=None, phi_layers=1):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("HybridAttention needs a CUDA device; there is no CPU fallback")
@@ -27,7 +28,8 @@ class HybridAttention:
         self.F = d if phi_dim is None else phi_dim
         self.rate = rate
         self._desc = binding.make_desc(B, H, N, d, grid, block, rate, phi_dim, poly_degree, softmax_scale,
-                                       stab_mode, kernel_path, softmax_idx)
+                                       stab_mode, kernel_path, softmax_idx, phi_layers=phi_layers,
+                                       phi_hidden=self.F if phi_layers == 2 else 0)
         self._h = binding.as_hybrid_attn_create(self._desc)
         self.workspace_bytes = binding.as_hybrid_attn_workspace_bytes(self._h)
         self.workspace_bytes_host = binding.as_hybrid_attn_workspace_bytes_host(self._h)
@@ -37,7 +39,7 @@ class HybridAttention:
     @classmethod
     def from_workload(cls, wl, **kw):
         return cls(wl.B, wl.H, wl.N, wl.d, wl.grid, wl.block, wl.rate, phi_dim=wl.F,
-                   poly_degree=wl.degree, **kw)
+                   poly_degree=wl.degree, phi_layers=getattr(wl, "layers", 1), **kw)
 
     @property
     def handle(self):
@@ -53,7 +55,7 @@ class HybridAttention:
     def softmax_indices(self):
         return binding.as_hybrid_attn_softmax_tokens(self._h)[1]
 
-    def forward(self, q, k, v, wq=None, wk=None, out=None, aux=None, stream=None):
+    def forward(self, q, k, v, wq=None, wk=None, out=None, aux=None, stream=None, wq2=None, wk2=None):
         import torch
         if out is None:
             out = torch.empty_like(q)
@@ -62,7 +64,8 @@ class HybridAttention:
         binding.as_hybrid_attn_forward(
             self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(),
             0 if wq is None else wq.data_ptr(), 0 if wk is None else wk.data_ptr(),
-            out.data_ptr(), 0 if aux is None else aux.data_ptr(), ws.data_ptr(), ws.numel(), st.cuda_stream)
+            out.data_ptr(), 0 if aux is None else aux.data_ptr(), ws.data_ptr(), ws.numel(), st.cuda_stream,
+            0 if wq2 is None else wq2.data_ptr(), 0 if wk2 is None else wk2.data_ptr())
         return out
 
     def forward_host(self, q_host, k_host, v_host, wq, wk, out_host, stream=None):

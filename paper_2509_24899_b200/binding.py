@@ -141,24 +141,26 @@ def as_hybrid_attn_workspace_bytes_host(h) -> int:
     return n.value
 
 
-def _weights(wq_ptr, wk_ptr):
+def _weights(wq_ptr, wk_ptr, wq2_ptr=0, wk2_ptr=0):
     if not wq_ptr and not wk_ptr:
         return None
     w = as_phi_weights_t()
     w.wq1, w.wk1 = wq_ptr, wk_ptr
+    w.wq2, w.wk2 = wq2_ptr or None, wk2_ptr or None
     return C.byref(w)
 
 
 def as_hybrid_attn_forward(h, q_ptr, k_ptr, v_ptr, wq_ptr, wk_ptr, out_ptr, aux_ptr, ws_ptr, ws_bytes,
-                           stream_ptr) -> None:
-    """All pointers are integer device addresses (e.g. tensor.data_ptr()); 0 / None means NULL."""
-    _check(lib().as_hybrid_attn_forward(h, q_ptr, k_ptr, v_ptr, _weights(wq_ptr, wk_ptr), out_ptr, aux_ptr or None,
+                           stream_ptr, wq2_ptr=0, wk2_ptr=0) -> None:
+    """All pointers are integer device addresses (e.g. tensor.data_ptr()); 0 / None means NULL.
+    wq2_ptr / wk2_ptr: second-layer weights of a two-layer feature map."""
+    _check(lib().as_hybrid_attn_forward(h, q_ptr, k_ptr, v_ptr, _weights(wq_ptr, wk_ptr, wq2_ptr, wk2_ptr), out_ptr, aux_ptr or None,
                                         ws_ptr, ws_bytes, stream_ptr or None), "as_hybrid_attn_forward")
 
 
 def as_hybrid_attn_forward_host(h, q_host, k_host, v_host, wq_ptr, wk_ptr, out_host, ws_ptr, ws_bytes,
-                                stream_ptr) -> None:
-    _check(lib().as_hybrid_attn_forward_host(h, q_host, k_host, v_host, _weights(wq_ptr, wk_ptr), out_host,
+                                stream_ptr, wq2_ptr=0, wk2_ptr=0) -> None:
+    _check(lib().as_hybrid_attn_forward_host(h, q_host, k_host, v_host, _weights(wq_ptr, wk_ptr, wq2_ptr, wk2_ptr), out_host,
                                              ws_ptr, ws_bytes, stream_ptr or None), "as_hybrid_attn_forward_host")
 
 

@@ -54,7 +54,9 @@ as_status_t validate(const as_hybrid_attn_desc_t* d) {
   // what this build has kernels for
   if (d->d != 64 && d->d != 128) return AS_ERR_UNSUPPORTED;
   if (d->phi_dim != d->d) return AS_ERR_UNSUPPORTED;
-  if (d->phi_layers != 1 || d->poly_degree > 2 || d->phi_act != AS_ACT_RELU) return AS_ERR_UNSUPPORTED;
+  if (d->phi_layers > 2 || d->poly_degree > 2 || d->phi_act != AS_ACT_RELU) return AS_ERR_UNSUPPORTED;
+  // two layers: hidden width equal to d, tensor-core path only
+  if (d->phi_layers == 2 && (d->phi_hidden != d->d || d->kernel_path != AS_PATH_TENSOR)) return AS_ERR_UNSUPPORTED;
   if ((long long)d->B * d->H > 65535) return AS_ERR_UNSUPPORTED;
   return AS_OK;
 }
@@ -74,6 +76,9 @@ void layout_workspace(as_hybrid_attn_s* h) {
   w.S = take(lin ? BH * d.phi_dim * d.d * 4 : 0);
   w.z = take(lin ? BH * d.phi_dim * 4 : 0);
   w.St = take(lin ? BH * d.phi_dim * d.d * 2 : 0);
+  const bool two = lin && d.phi_layers == 2;
+  w.h1q = take(two ? BH * (size_t)d.N * d.phi_hidden * 2 : 0);
+  w.h1k = take(two ? BH * (size_t)d.N * d.phi_hidden * 2 : 0);
   w.total = std::max<size_t>(off, 256);
   const size_t t = BH * d.N * d.d * 2;
   off = w.total;
@@ -203,8 +208,10 @@ as_status_t as_hybrid_attn_forward(as_hybrid_attn_t h, const void* q, const void
   const bool lin = h->n_l > 0;
   if (lin) {
     if (!w || !w->wq1 || !w->wk1) return AS_ERR_INVALID_ARG;
-    if (w->bq1 || w->bk1 || w->wq2 || w->wk2 || w->bq2 || w->bk2) return AS_ERR_UNSUPPORTED;
-    if (((uintptr_t)w->wq1 | (uintptr_t)w->wk1) & 15) return AS_ERR_INVALID_ARG;
+    if (w->bq1 || w->bk1 || w->bq2 || w->bk2) return AS_ERR_UNSUPPORTED;
+    if (d.phi_layers == 1 && (w->wq2 || w->wk2)) return AS_ERR_INVALID_ARG;
+    if (d.phi_layers == 2 && (!w->wq2 || !w->wk2)) return AS_ERR_INVALID_ARG;
+    if (((uintptr_t)w->wq1 | (uintptr_t)w->wk1 | (uintptr_t)w->wq2 | (uintptr_t)w->wk2) & 15) return AS_ERR_INVALID_ARG;
   }
   if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15) return AS_ERR_INVALID_ARG;
   if (aux && ((uintptr_t)aux & 3)) return AS_ERR_INVALID_ARG;
@@ -216,6 +223,12 @@ as_status_t as_hybrid_attn_forward(as_hybrid_attn_t h, const void* q, const void
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;
   a.wq = lin ? (const __nv_bfloat16*)w->wq1 : nullptr;
   a.wk = lin ? (const __nv_bfloat16*)w->wk1 : nullptr;
+  const bool two = lin && d.phi_layers == 2;
+  a.wq2 = two ? (const __nv_bfloat16*)w->wq2 : nullptr;
+  a.wk2 = two ? (const __nv_bfloat16*)w->wk2 : nullptr;
+  a.h1q = two ? (__nv_bfloat16*)(ws + h->ws.h1q) : nullptr;
+  a.h1k = two ? (__nv_bfloat16*)(ws + h->ws.h1k) : nullptr;
+  a.layers = d.phi_layers;
   a.out = (__nv_bfloat16*)out; a.aux = aux;
   const bool compact = h->n_s > 0 && lin;
   a.ks_w = compact ? (__nv_bfloat16*)(ws + h->ws.ks) : nullptr;
@@ -232,6 +245,11 @@ as_status_t as_hybrid_attn_forward(as_hybrid_attn_t h, const void* q, const void
 
   const bool simt = d.kernel_path == AS_PATH_SIMT;
   cudaError_t e = cudaSuccess;
+  if (two) {
+    { ProfileScope p(h, st, AS_KERNEL_KPASS);     // counted with the K pass: it feeds it
+      e = as_tensor_phi1(a, st); }
+    if (e != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
+  }
   if (lin) {
     { ProfileScope p(h, st, AS_KERNEL_KPASS);
       e = simt ? as_simt_kpass(a, st) : as_tensor_kpass(a, st); }

@@ -18,6 +18,7 @@ struct as_ws_layout {
   size_t part_s = 0, part_z = 0;        // per-chunk partial state   [B*H, chunks, F, d] / [.., F] fp32
   size_t S = 0, z = 0;                  // final state               [B*H, F, d] / [B*H, F] fp32
   size_t St = 0;                        // S transposed              [B*H, d, F] bf16 (MMA operand)
+  size_t h1q = 0, h1k = 0;              // first-layer activations   [B*H, N, hidden] bf16 (two-layer feature map only)
   size_t total = 0;
   size_t stage_q = 0, stage_k = 0, stage_v = 0, stage_o = 0, total_host = 0;
 };
@@ -25,6 +26,9 @@ struct as_ws_layout {
 // Everything a kernel launch needs, resolved to device pointers.
 struct as_launch_args {
   const __nv_bfloat16 *q, *k, *v, *wq, *wk;
+  const __nv_bfloat16 *wq2, *wk2;       // second feature-map layer [H, F, hidden] (NULL for a one-layer map)
+  __nv_bfloat16 *h1q, *h1k;             // relu(q W_q1^T), relu(k W_k1^T) when the map has two layers
+  int layers;                           // depth of the feature map's embedding network (1 or 2)
   __nv_bfloat16* out;
   float* aux;
   const __nv_bfloat16 *ks, *vs;         // softmax keys / values the Q pass reads (k, v themselves at R = 1)
@@ -64,6 +68,8 @@ cudaError_t as_simt_qpass(const as_launch_args& a, cudaStream_t st);
 cudaError_t as_reduce_state(const as_launch_args& a, cudaStream_t st);
 cudaError_t as_tensor_kpass(const as_launch_args& a, cudaStream_t st);
 cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st);
+// First layer of a two-layer feature map for q and k in one launch: h1 = relu(x W1^T).
+cudaError_t as_tensor_phi1(const as_launch_args& a, cudaStream_t st);
 // One-time set-up of the tensor path on the current device (driver entry points, smem opt-in).
 cudaError_t as_tensor_init();
 

@@ -32,6 +32,7 @@ constexpr int BOX_BYTES = 128 * 128;     // one TMA box: 128 rows x 64 bf16 (128
 // ======================================================================================
 struct QParams {
   int N, n_s, nkv, lin, stab_mode, P, H;
+  int layers;                // depth of the feature map: with 2, tmH holds relu(q W_1^T) and tmW is W_2
   float scale_log2;          // softmax scale * log2(e)
   const float* z;            // [B*H][F]
   float* aux;                // [B*H][N][3] or nullptr
@@ -96,7 +97,7 @@ __global__ void __launch_bounds__(Q_THREADS, 1)
 qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
              const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmW,
              const __grid_constant__ CUtensorMap tmSt, const __grid_constant__ CUtensorMap tmO,
-             const QParams p) {
+             const __grid_constant__ CUtensorMap tmH, const QParams p) {
   using L = QLayout<D>;
   constexpr int F = D;
   extern __shared__ uint8_t smem_raw[];
@@ -141,7 +142,10 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   const uint32_t tO[2] = {tmem + 256u, tmem + 384u};
   const uint32_t sQ[2] = {sbase + L::Q_OFF, sbase + L::Q_OFF + L::TILE};
   auto sKV = [&](int item) { return sbase + L::KV_OFF + (item % KV_STAGES) * L::TILE; };
-  const int n_items = 2 * nkv + (p.lin ? 2 : 0);
+  // items of the K/V ring: K and V tiles alternating, then for the linear tail the last-layer weights,
+  // (with a two-layer feature map) the two groups' first-layer activations, and S^T
+  const int it_w = 2 * nkv, it_h = 2 * nkv + 1, it_st = 2 * nkv + (p.layers == 2 ? 3 : 1);
+  const int n_items = p.lin ? it_st + 1 : 2 * nkv;
 
   if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
@@ -160,8 +164,10 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         if (it < 2 * nkv) {
           const int j = it >> 1;
           load_tile<D>(sKV(it), (it & 1) ? &tmV : &tmK, bar(B_FULL + st), j * 128, bh);
-        } else if (it == 2 * nkv) {
+        } else if (it == it_w) {
           load_tile<D>(sKV(it), &tmW, bar(B_FULL + st), 0, h);          // W_q[h]: [F rows][D]
+        } else if (it < it_st) {
+          load_tile<D>(sKV(it), &tmH, bar(B_FULL + st), row0 + (it - it_h) * 128, bh);   // relu(q W_1^T) of group it - it_h
         } else {
           load_tile<D>(sKV(it), &tmSt, bar(B_FULL + st), 0, bh);        // S^T[bh]: [D rows][F]
         }
@@ -230,21 +236,25 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       }
     }
     if (ok && p.lin) {
-      ok = full_wait(2 * nkv);
-      if (ok) {
+      ok = full_wait(it_w);
+      for (int g = 0; ok && g < 2; ++g) {
+        // Phi = X W^T with X = Q (one layer) or the first-layer activations (two layers)
+        if (p.layers == 2) ok = full_wait(it_h + g);
+        if (!ok) break;
         tc_fence_after();
         if (lane == 0) {
-          for (int g = 0; g < 2; ++g) { issue_kmajor<D>(tS[g], kmajor_desc(sQ[g]), kmajor_desc(sKV(2 * nkv)), ID_PHI, false); tc_commit(bar(B_S + g)); }
+          issue_kmajor<D>(tS[g], kmajor_desc(p.layers == 2 ? sKV(it_h + g) : sQ[g]), kmajor_desc(sKV(it_w)), ID_PHI, false);
+          tc_commit(bar(B_S + g));
         }
         __syncwarp();
-        ok = full_wait(2 * nkv + 1);
       }
+      if (ok) ok = full_wait(it_st);
       for (int g = 0; ok && g < 2; ++g) {
         ok = mbar_wait_warp(bar(B_P + g), nkv & 1, wc);
         if (!ok) break;
         tc_fence_after();
         if (lane == 0) {
-          issue_kmajor<F>(tO[g], kmajor_desc(sQ[g]), kmajor_desc(sKV(2 * nkv + 1)), ID_LIN, nkv > 0);
+          issue_kmajor<F>(tO[g], kmajor_desc(sQ[g]), kmajor_desc(sKV(it_st)), ID_LIN, nkv > 0);
           tc_commit(bar(B_O + g));
         }
         __syncwarp();
@@ -414,24 +424,30 @@ struct KParams {
 };
 
 constexpr int K_THREADS = 256;           // warps 0-3: feature warps; 4: TMA; 5: MMA; 6-7: gather
-constexpr int K_STAGES = 3;
+// stages of the K / V ring: 3 with a one-layer feature map; 2 with two layers, where every stage also holds
+// the tile of first-layer activations
+template <int LAYERS> constexpr int k_stages() { return LAYERS == 2 ? 2 : 3; }
 
-template <int D>
+template <int D, int LAYERS>
 struct KLayout {
+  static constexpr int K_STAGES = k_stages<LAYERS>();
+  static constexpr int STAGE_TILES = LAYERS == 2 ? 3 : 2;        // K tile, V tile (, first-layer activations)
   static constexpr int TILE = 128 * D * 2;
-  static constexpr int W_OFF = 0;                                // W_k as a [128 x D] tile (rows >= F are zero)
-  static constexpr int KV_OFF = TILE;                            // K_STAGES x (K tile, V tile)
-  static constexpr int BAR_OFF = KV_OFF + K_STAGES * 2 * TILE;
+  static constexpr int W_OFF = 0;                                // last-layer weights as a [128 x D] tile (rows >= F are zero)
+  static constexpr int KV_OFF = TILE;                            // K_STAGES x STAGE_TILES tiles
+  static constexpr int BAR_OFF = KV_OFF + K_STAGES * STAGE_TILES * TILE;
   static constexpr int MASK_OFF = BAR_OFF + 256;                 // 2 x 4 words: linear-token bits per tile
   static constexpr int RANK_OFF = MASK_OFF + 64;                 // K_STAGES x 128 int32
   static constexpr int TOTAL = RANK_OFF + K_STAGES * 512 + 1024;
 };
 
-template <int D>
+// LAYERS == 2: the features are phi(relu(k W_1^T) W_2^T); relu(k W_1^T) comes precomputed (tmH), tmW is W_2.
+template <int D, int LAYERS>
 __global__ void __launch_bounds__(K_THREADS, 1)
 kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-             const __grid_constant__ CUtensorMap tmW, const KParams p) {
-  using L = KLayout<D>;
+             const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH, const KParams p) {
+  using L = KLayout<D, LAYERS>;
+  constexpr int K_STAGES = L::K_STAGES;
   constexpr int F = D;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -474,8 +490,9 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   const uint32_t tD1[2] = {tmem + 0u, tmem + 128u};
   const uint32_t tAcc = tmem + 256u;
   const uint32_t sW = sbase + L::W_OFF;
-  auto sK = [&](int st) { return sbase + L::KV_OFF + st * 2 * L::TILE; };
-  auto sV = [&](int st) { return sbase + L::KV_OFF + st * 2 * L::TILE + L::TILE; };
+  auto sK = [&](int st) { return sbase + L::KV_OFF + st * L::STAGE_TILES * L::TILE; };
+  auto sV = [&](int st) { return sbase + L::KV_OFF + st * L::STAGE_TILES * L::TILE + L::TILE; };
+  auto sH = [&](int st) { return sbase + L::KV_OFF + st * L::STAGE_TILES * L::TILE + 2 * L::TILE; };   // two layers only
 
   if (warp == 4) {
     // ------------------------------------------------------------ TMA producer
@@ -488,7 +505,8 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       const int st = t % K_STAGES, use = t / K_STAGES;
       if (!mbar_wait_warp(bar(B_EMPTY + st), (use & 1) ^ 1, wc)) break;
       if (lane == 0) {
-        mbar_expect_tx(bar(B_FULL + st), 2 * L::TILE);
+        mbar_expect_tx(bar(B_FULL + st), L::STAGE_TILES * L::TILE);
+        if (LAYERS == 2) load_tile<D>(sH(st), &tmH, bar(B_FULL + st), (t_begin + t) * 128, bh);
         load_tile<D>(sK(st), &tmK, bar(B_FULL + st), (t_begin + t) * 128, bh);
         load_tile<D>(sV(st), &tmV, bar(B_FULL + st), (t_begin + t) * 128, bh);
       }
@@ -506,7 +524,7 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         if (!ok) break;
         tc_fence_after();
         if (lane == 0) {
-          issue_kmajor<D>(tD1[t & 1], kmajor_desc(sW), kmajor_desc(sK(st)), ID_PHI, false);
+          issue_kmajor<D>(tD1[t & 1], kmajor_desc(sW), kmajor_desc(LAYERS == 2 ? sH(st) : sK(st)), ID_PHI, false);
           tc_commit(bar(B_D1 + (t & 1)));
         }
         __syncwarp();
@@ -544,7 +562,7 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       load_ranks(t + 1, rk_next);
       if (!mbar_wait_warp(bar(B_FULL + st), (t / K_STAGES) & 1, wc)) break;
       if (p.ks_w != nullptr) {
-        const uint8_t* kt = smem + L::KV_OFF + st * 2 * L::TILE;
+        const uint8_t* kt = smem + L::KV_OFF + st * L::STAGE_TILES * L::TILE;
         const uint8_t* vt = kt + L::TILE;
         constexpr int CH = D / 8;                          // 16-byte chunks per row
         for (int e = 0; e < 2; ++e) {
@@ -647,6 +665,108 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 }
 
 // ======================================================================================
+// First layer of a two-layer feature map ("Characterization of phi": the embedding network): h1 = relu(x W_1^T)
+// for x = q (blockIdx.z == 0) and x = k (blockIdx.z == 1).  One 128-token tile per CTA.
+// ======================================================================================
+struct P1Params { int H; uint32_t* status; };
+constexpr int P1_THREADS = 160;          // warps 0-3: epilogue (one thread per token row); warp 4: TMA + MMA
+
+template <int D>
+struct P1Layout {
+  static constexpr int TILE = 128 * D * 2;
+  static constexpr int X_OFF = 0, W_OFF = TILE, BAR_OFF = 2 * TILE;
+  static constexpr int TOTAL = BAR_OFF + 64 + 1024;
+};
+
+template <int D>
+__global__ void __launch_bounds__(P1_THREADS)
+phi1_kernel(const __grid_constant__ CUtensorMap tmXq, const __grid_constant__ CUtensorMap tmXk,
+            const __grid_constant__ CUtensorMap tmWq, const __grid_constant__ CUtensorMap tmWk,
+            const __grid_constant__ CUtensorMap tmHq, const __grid_constant__ CUtensorMap tmHk, const P1Params p) {
+  using L = P1Layout<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::BAR_OFF);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::BAR_OFF + 16);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::BAR_OFF + 20);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = blockIdx.y, h = bh % p.H, row0 = blockIdx.x * 128;
+  const bool is_k = blockIdx.z != 0;
+  const CUtensorMap* tmX = is_k ? &tmXk : &tmXq;
+  const CUtensorMap* tmW = is_k ? &tmWk : &tmWq;
+  const CUtensorMap* tmH = is_k ? &tmHk : &tmHq;
+  const WaitCtx wc{p.status, abort_flag};
+  const uint32_t bar_full = smem_u32(bars), bar_done = smem_u32(bars + 1);
+
+  __shared__ uint32_t s_skip;
+  if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile uint32_t*>(p.status);
+  __syncthreads();
+  if (s_skip != 0u) return;
+  if (threadIdx.x == 0) {
+    *abort_flag = 0u;
+    mbar_init(bar_full, 1); mbar_init(bar_done, 1);
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 4) { tmem_alloc(smem_u32(tmem_slot), 128); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t sX = sbase + L::X_OFF, sW = sbase + L::W_OFF;
+
+  if (warp == 4) {
+    if (lane == 0) {
+      mbar_expect_tx(bar_full, 2 * L::TILE);
+      load_tile<D>(sX, tmX, bar_full, row0, bh);
+      load_tile<D>(sW, tmW, bar_full, 0, h);                  // W_1[h]: [hidden rows][D]
+    }
+    __syncwarp();
+    if (mbar_wait_warp(bar_full, 0, wc)) {
+      tc_fence_after();
+      if (lane == 0) {
+        issue_kmajor<D>(tmem, kmajor_desc(sX), kmajor_desc(sW), make_idesc(128, D, 0, 0), false);   // X W_1^T, N = hidden = D
+        tc_commit(bar_done);
+      }
+      __syncwarp();
+    }
+  } else {
+    const int r = warp * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    bool ok = mbar_wait_warp(bar_done, 0, wc);
+    if (ok) {
+      tc_fence_after();
+      uint32_t x[32];
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        tmem_ld32(tmem + lane_off + c * 32, x);
+        tmem_ld_wait(x);
+        uint32_t w[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          w[i] = pack_bf16(fmaxf(__uint_as_float(x[2 * i]), 0.f), fmaxf(__uint_as_float(x[2 * i + 1]), 0.f));
+        store_row_chunk(smem + L::X_OFF, r, c * 32, w);       // the X tile has been consumed by the MMA
+      }
+      fence_proxy_async();
+    }
+    named_barrier_sync(1, 128);                               // reached by every epilogue thread, also after a failed wait
+    if (ok && r == 0) {
+#pragma unroll
+      for (int b = 0; b < D / 64; ++b) tma_store_3d(tmH, sX + b * BOX_BYTES, b * 64, row0, bh);
+      tma_store_commit();
+      tma_store_wait_all();
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 128);
+  }
+}
+
+// ======================================================================================
 // Host side: tensor maps and launches
 // ======================================================================================
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -690,25 +810,51 @@ cudaError_t as_tensor_init() {
   cudaError_t e;
   if ((e = opt_in_smem(qpass_kernel<128>, QLayout<128>::TOTAL)) != cudaSuccess) return e;
   if ((e = opt_in_smem(qpass_kernel<64>, QLayout<64>::TOTAL)) != cudaSuccess) return e;
-  if ((e = opt_in_smem(kpass_kernel<128>, KLayout<128>::TOTAL)) != cudaSuccess) return e;
-  if ((e = opt_in_smem(kpass_kernel<64>, KLayout<64>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(kpass_kernel<128, 1>, KLayout<128, 1>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(kpass_kernel<64, 1>, KLayout<64, 1>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(phi1_kernel<128>, P1Layout<128>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(phi1_kernel<64>, P1Layout<64>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(kpass_kernel<128, 2>, KLayout<128, 2>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(kpass_kernel<64, 2>, KLayout<64, 2>::TOTAL)) != cudaSuccess) return e;
   return cudaSuccess;
+}
+
+cudaError_t as_tensor_phi1(const as_launch_args& a, cudaStream_t st) {
+  if (g_encode == nullptr) return cudaErrorNotSupported;
+  const int BH = a.B * a.H;
+  CUtensorMap tmXq, tmXk, tmWq, tmWk, tmHq, tmHk;
+  if (!make_map(&tmXq, a.q, a.d, a.N, BH, 128) || !make_map(&tmXk, a.k, a.d, a.N, BH, 128) ||
+      !make_map(&tmWq, a.wq, a.d, a.d, a.H, 128) || !make_map(&tmWk, a.wk, a.d, a.d, a.H, 128) ||
+      !make_map(&tmHq, a.h1q, a.d, a.N, BH, 128) || !make_map(&tmHk, a.h1k, a.d, a.N, BH, 128))
+    return cudaErrorInvalidValue;
+  P1Params p{a.H, a.status};
+  dim3 grid((a.N + 127) / 128, BH, 2);
+  if (a.d == 128) phi1_kernel<128><<<grid, P1_THREADS, P1Layout<128>::TOTAL, st>>>(tmXq, tmXk, tmWq, tmWk, tmHq, tmHk, p);
+  else phi1_kernel<64><<<grid, P1_THREADS, P1Layout<64>::TOTAL, st>>>(tmXq, tmXk, tmWq, tmWk, tmHq, tmHk, p);
+  return cudaGetLastError();
 }
 
 cudaError_t as_tensor_kpass(const as_launch_args& a, cudaStream_t st) {
   if (g_encode == nullptr) return cudaErrorNotSupported;
   const int BH = a.B * a.H;
-  CUtensorMap tmK, tmV, tmW;
+  CUtensorMap tmK, tmV, tmW, tmH;
   if (!make_map(&tmK, a.k, a.d, a.N, BH, 128) || !make_map(&tmV, a.v, a.d, a.N, BH, 128) ||
-      !make_map(&tmW, a.wk, a.d, a.F, a.H, 128))
+      !make_map(&tmW, a.layers == 2 ? a.wk2 : a.wk, a.d, a.F, a.H, 128))
     return cudaErrorInvalidValue;
+  if (a.layers == 2) { if (!make_map(&tmH, a.h1k, a.d, a.N, BH, 128)) return cudaErrorInvalidValue; }
+  else tmH = tmK;               // never used with a one-layer map
   KParams p{};
   p.N = a.N; p.n_s = a.n_s; p.n_chunks = a.n_chunks; p.chunk_tiles = a.chunk_tiles; p.P = a.P; p.F = a.F;
   p.H = a.H; p.sm_rank = a.sm_rank; p.ks_w = a.ks_w; p.vs_w = a.vs_w; p.k = a.k; p.v = a.v;
   p.part_s = a.part_s; p.part_z = a.part_z; p.status = a.status;
   dim3 grid(a.n_chunks, BH, 1);
-  if (a.d == 128) kpass_kernel<128><<<grid, K_THREADS, KLayout<128>::TOTAL, st>>>(tmK, tmV, tmW, p);
-  else kpass_kernel<64><<<grid, K_THREADS, KLayout<64>::TOTAL, st>>>(tmK, tmV, tmW, p);
+  if (a.layers == 2) {
+    if (a.d == 128) kpass_kernel<128, 2><<<grid, K_THREADS, KLayout<128, 2>::TOTAL, st>>>(tmK, tmV, tmW, tmH, p);
+    else kpass_kernel<64, 2><<<grid, K_THREADS, KLayout<64, 2>::TOTAL, st>>>(tmK, tmV, tmW, tmH, p);
+  } else {
+    if (a.d == 128) kpass_kernel<128, 1><<<grid, K_THREADS, KLayout<128, 1>::TOTAL, st>>>(tmK, tmV, tmW, tmH, p);
+    else kpass_kernel<64, 1><<<grid, K_THREADS, KLayout<64, 1>::TOTAL, st>>>(tmK, tmV, tmW, tmH, p);
+  }
   return cudaGetLastError();
 }
 
@@ -716,7 +862,7 @@ cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st) {
   if (g_encode == nullptr) return cudaErrorNotSupported;
   const int BH = a.B * a.H;
   const bool lin = a.n_l > 0;
-  CUtensorMap tmQ, tmK, tmV, tmW, tmSt, tmO;
+  CUtensorMap tmQ, tmK, tmV, tmW, tmSt, tmO, tmH;
   if (!make_map(&tmQ, a.q, a.d, a.N, BH, 128) || !make_map(&tmO, a.out, a.d, a.N, BH, 128)) return cudaErrorInvalidValue;
   if (a.n_s > 0) {
     if (!make_map(&tmK, a.ks, a.d, a.n_s, BH, 128) || !make_map(&tmV, a.vs, a.d, a.n_s, BH, 128)) return cudaErrorInvalidValue;
@@ -725,17 +871,20 @@ cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st) {
   }
   if (lin) {
     // boxes are always 128 rows: rows past F (or d) are out of bounds and arrive as zeros
-    if (!make_map(&tmW, a.wq, a.d, a.F, a.H, 128) || !make_map(&tmSt, a.St, a.F, a.d, BH, 128)) return cudaErrorInvalidValue;
+    if (!make_map(&tmW, a.layers == 2 ? a.wq2 : a.wq, a.d, a.F, a.H, 128) || !make_map(&tmSt, a.St, a.F, a.d, BH, 128)) return cudaErrorInvalidValue;
   } else {
     tmW = tmQ; tmSt = tmQ;      // never used: no linear branch at rate 1
   }
+  if (lin && a.layers == 2) { if (!make_map(&tmH, a.h1q, a.d, a.N, BH, 128)) return cudaErrorInvalidValue; }
+  else tmH = tmQ;             // never used with a one-layer map
   QParams p{};
+  p.layers = lin ? a.layers : 1;
   p.N = a.N; p.n_s = a.n_s; p.nkv = (a.n_s + 127) / 128; p.lin = lin ? 1 : 0; p.stab_mode = a.stab_mode; p.P = a.P;
   p.H = a.H;
   p.scale_log2 = a.scale * 1.4426950408889634f;
   p.z = a.z; p.aux = a.aux; p.status = a.status;
   dim3 grid((a.N + 255) / 256, BH, 1);
-  if (a.d == 128) qpass_kernel<128><<<grid, Q_THREADS, QLayout<128>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmO, p);
-  else qpass_kernel<64><<<grid, Q_THREADS, QLayout<64>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmO, p);
+  if (a.d == 128) qpass_kernel<128><<<grid, Q_THREADS, QLayout<128>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmO, tmH, p);
+  else qpass_kernel<64><<<grid, Q_THREADS, QLayout<64>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmO, tmH, p);
   return cudaGetLastError();
 }

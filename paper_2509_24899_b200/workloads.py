@@ -34,6 +34,7 @@ class Workload:
     seed: int
     rms_norm_qk: bool = True
     degree: int = 2      # polynomial degree P of the feature map
+    layers: int = 1      # depth of the feature map's embedding network (2: hidden width = F)
 
     @property
     def N(self) -> int:
@@ -104,7 +105,7 @@ def bf16_bits_to_f64(b: np.ndarray) -> np.ndarray:
 def generate(wl: Workload, wq_gain: float = 1.0, heads: int | None = None):
     """Draw one layer's inputs.  Returns a dict of uint16 arrays holding bf16 bit patterns:
 
-      q, k, v : [B, H, N, d]      wq, wk : [H, F, d]
+      q, k, v : [B, H, N, d]      wq, wk : [H, F, d]      (wl.layers == 2: also wq2, wk2 : [H, F, F])
 
     Draw order is Q, K, V, W_q, W_k from numpy's PCG64 seeded with `wl.seed`.
     `wq_gain` multiplies W_q before rounding (used by the tests to make the softmax and
@@ -125,9 +126,16 @@ def generate(wl: Workload, wq_gain: float = 1.0, heads: int | None = None):
     wk = rng.uniform(-a, a, size=(wl.H, wl.F, wl.d)).astype(np.float32)
     out["wq"] = f32_to_bf16_bits(wq * np.float32(wq_gain))
     out["wk"] = f32_to_bf16_bits(wk)
+    weight_names = ["wq", "wk"]
+    if wl.layers == 2:
+        # second layer [H, F, hidden] with hidden = F, drawn after the first layers (which then map d -> hidden)
+        a2 = math.sqrt(6.0 / (wl.F + wl.F))
+        out["wq2"] = f32_to_bf16_bits(rng.uniform(-a2, a2, size=(wl.H, wl.F, wl.F)).astype(np.float32))
+        out["wk2"] = f32_to_bf16_bits(rng.uniform(-a2, a2, size=(wl.H, wl.F, wl.F)).astype(np.float32))
+        weight_names += ["wq2", "wk2"]
     if heads is not None and heads < wl.H:
         for name in ("q", "k", "v"):
             out[name] = np.ascontiguousarray(out[name][:, :heads])
-        out["wq"] = np.ascontiguousarray(out["wq"][:heads])
-        out["wk"] = np.ascontiguousarray(out["wk"][:heads])
+        for name in weight_names:
+            out[name] = np.ascontiguousarray(out[name][:heads])
     return out

@@ -327,3 +327,73 @@ def test_gpu_argument_errors():
         binding.as_hybrid_attn_forward(op.handle, data["q"].data_ptr(), data["k"].data_ptr(), data["v"].data_ptr(),
                                        0, 0, out.data_ptr(), 0, ws.data_ptr(), op.workspace_bytes, 0)
     assert e.value.status == binding.AS_ERR_INVALID_ARG
+
+
+TWO_LAYER = {
+    "two_layer_d128": W.Workload("two_layer_d128", B=1, H=2, d=128, F=128, grid=(3, 10, 13), block=(1, 6, 8),
+                                 rate=4, seed=31, layers=2),
+    "two_layer_d64": W.Workload("two_layer_d64", B=2, H=3, d=64, F=64, grid=(2, 9, 31), block=(1, 4, 4),
+                                rate=2, seed=32, rms_norm_qk=False, layers=2),
+    "two_layer_rate0": W.Workload("two_layer_rate0", B=1, H=2, d=128, F=128, grid=(3, 10, 13), block=(1, 6, 8),
+                                  rate=0, seed=33, layers=2),
+    "two_layer_chunks": W.Workload("two_layer_chunks", B=1, H=1, d=128, F=128, grid=(8, 30, 52), block=(1, 6, 8),
+                                   rate=8, seed=34, layers=2),
+}
+
+
+def _oracle_two_layer(wl, d64, mode, rows=None):
+    """Oracle with the two-layer embedding network: the weights of a head are the list [W_1, W_2]."""
+    mask = oracle_mask(wl)
+    B, H = d64["q"].shape[:2]
+    n_rows = wl.N if rows is None else len(rows)
+    y = np.empty((B, H, n_rows, wl.d))
+    aux = np.empty((B, H, n_rows, 3))
+    S = np.empty((B, H, wl.F, wl.d))
+    z = np.empty((B, H, wl.F))
+    for b in range(B):
+        for h in range(H):
+            wq, wk = [d64["wq"][h], d64["wq2"][h]], [d64["wk"][h], d64["wk2"][h]]
+            y[b, h], aux[b, h] = O.hybrid_attention_head(d64["q"][b, h], d64["k"][b, h], d64["v"][b, h], wq, wk, mask,
+                                                         None, mode, wl.degree, rows=rows)
+            if not mask.all():
+                S[b, h], z[b, h] = O.linear_state(d64["k"][b, h], d64["v"][b, h], wk, mask, wl.degree)
+    return y, aux, S, z
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("name", sorted(TWO_LAYER))
+def test_two_layer_feature_map(mode, name):
+    """phi(x) = poly(ReLU(W_2 ReLU(W_1 x))): first layer by its own kernel, second layer fused into the K and Q pass."""
+    import torch
+    from paper_2509_24899_b200 import HybridAttention
+    wl = TWO_LAYER[name]
+    data = W.generate(wl, wq_gain=0.05 if wl.rate else 1.0)
+    dev = {k: to_cuda_bf16(v) for k, v in data.items()}
+    op = HybridAttention.from_workload(wl, stab_mode=mode)
+    aux = torch.full((wl.B, wl.H, wl.N, 3), float("nan"), dtype=torch.float32, device="cuda")
+    out = op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], aux=aux, wq2=dev["wq2"], wk2=dev["wk2"])
+    Sg, zg = op.linear_state()
+    torch.cuda.synchronize()
+    assert op.last_status() == 0
+    d64 = oracle_inputs(data)
+    ref, ref_aux, S, z = _oracle_two_layer(wl, d64, mode)
+    assert errors(Sg.cpu().numpy().astype(np.float64), S)[0] <= 5e-3
+    assert errors(zg.cpu().numpy().astype(np.float64), z)[0] <= 5e-3
+    got = from_cuda_bf16(out)
+    ok = np.isfinite(ref).all(-1)
+    assert ok.mean() > 0.99
+    assert_parity(got[ok], ref[ok], name, strict=False)
+    _check_aux(aux.cpu().numpy().astype(np.float64)[ok], ref_aux[ok], wl, op.n_softmax)
+
+
+def test_two_layer_needs_its_second_weights_and_the_tensor_path():
+    from paper_2509_24899_b200 import HybridAttention, binding, AsError, AS_PATH_SIMT
+    wl = TWO_LAYER["two_layer_d128"]
+    with pytest.raises(AsError) as e:
+        HybridAttention.from_workload(wl, kernel_path=AS_PATH_SIMT)
+    assert e.value.status == binding.AS_ERR_UNSUPPORTED
+    op = HybridAttention.from_workload(wl)
+    dev = {k: to_cuda_bf16(v) for k, v in W.generate(wl).items()}
+    with pytest.raises(AsError) as e:
+        op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"])
+    assert e.value.status == binding.AS_ERR_INVALID_ARG
