@@ -75,7 +75,7 @@ void layout_workspace(as_hybrid_attn_s* h) {
   w.part_z = take(lin ? BH * h->n_chunks * d.phi_dim * 4 : 0);
   w.S = take(lin ? BH * d.phi_dim * d.d * 4 : 0);
   w.z = take(lin ? BH * d.phi_dim * 4 : 0);
-  w.St = take(lin ? BH * d.phi_dim * d.d * 2 : 0);
+  w.Sb = take(lin ? BH * d.phi_dim * d.d * 2 : 0);
   const bool two = lin && d.phi_layers == 2;
   w.h1q = take(two ? BH * (size_t)d.N * d.phi_hidden * 2 : 0);
   w.h1k = take(two ? BH * (size_t)d.N * d.phi_hidden * 2 : 0);
@@ -237,7 +237,7 @@ as_status_t as_hybrid_attn_forward(as_hybrid_attn_t h, const void* q, const void
   a.vs = compact ? a.vs_w : a.v;
   a.part_s = (float*)(ws + h->ws.part_s); a.part_z = (float*)(ws + h->ws.part_z);
   a.S = (float*)(ws + h->ws.S); a.z = (float*)(ws + h->ws.z);
-  a.St = (__nv_bfloat16*)(ws + h->ws.St);
+  a.Sb = (__nv_bfloat16*)(ws + h->ws.Sb);
   a.sm_rank = h->d_sm_rank; a.status = h->d_status;
   a.B = d.B; a.H = d.H; a.N = d.N; a.d = d.d; a.F = d.phi_dim; a.P = d.poly_degree;
   a.n_s = h->n_s; a.n_l = h->n_l; a.n_chunks = h->n_chunks; a.chunk_tiles = h->chunk_tiles;

@@ -17,7 +17,7 @@ struct as_ws_layout {
   size_t ks = 0, vs = 0;                // compacted softmax K / V   [B*H, N_S, d] bf16
   size_t part_s = 0, part_z = 0;        // per-chunk partial state   [B*H, chunks, F, d] / [.., F] fp32
   size_t S = 0, z = 0;                  // final state               [B*H, F, d] / [B*H, F] fp32
-  size_t St = 0;                        // S transposed              [B*H, d, F] bf16 (MMA operand)
+  size_t Sb = 0;                        // S rounded to bf16         [B*H, F, d] (MMA operand of the Q pass)
   size_t h1q = 0, h1k = 0;              // first-layer activations   [B*H, N, hidden] bf16 (two-layer feature map only)
   size_t total = 0;
   size_t stage_q = 0, stage_k = 0, stage_v = 0, stage_o = 0, total_host = 0;
@@ -34,7 +34,7 @@ struct as_launch_args {
   const __nv_bfloat16 *ks, *vs;         // softmax keys / values the Q pass reads (k, v themselves at R = 1)
   __nv_bfloat16 *ks_w, *vs_w;           // where the K pass writes the compacted rows (NULL at R = 1)
   float *part_s, *part_z, *S, *z;
-  __nv_bfloat16* St;
+  __nv_bfloat16* Sb;
   const int32_t* sm_rank;               // [N]: position in T_S, or -1 for a linear token
   uint32_t* status;                     // device status word
   int B, H, N, d, F, P;

@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(KP_THREADS) simt_kpass_kernel(as_launch_args a
 }
 
 // Sums the per-chunk partial states in chunk order (deterministic) and writes S, z in fp32 and
-// S transposed in bf16 ([d][F], the K-major MMA operand of the tensor path).
+// S rounded to bf16 (same [F][d] layout: the tensor path reads it like a V tile).
 __global__ void reduce_state_kernel(as_launch_args a) {
   const int bh = blockIdx.y;
   const int D = a.d, F = a.F;
@@ -107,8 +107,7 @@ __global__ void reduce_state_kernel(as_launch_args a) {
     float s = 0.f;
     for (int c = 0; c < a.n_chunks; ++c) s += a.part_s[((size_t)bh * a.n_chunks + c) * F * D + i];
     a.S[(size_t)bh * F * D + i] = s;
-    const int f = i / D, dd = i % D;
-    a.St[(size_t)bh * F * D + (size_t)dd * F + f] = __float2bfloat16_rn(s);
+    a.Sb[(size_t)bh * F * D + i] = __float2bfloat16_rn(s);
   } else if (i < F * D + F) {
     const int f = i - F * D;
     float s = 0.f;

@@ -93,6 +93,8 @@ AS_DEV void tma_store_3d(const CUtensorMap* m, uint32_t src, int x, int y, int z
 }
 AS_DEV void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 AS_DEV void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Only until the sources of all committed stores have been read: the shared memory can be reused.
+AS_DEV void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
 // ---------------------------------------------------------------- tensor memory
 AS_DEV void tmem_alloc(uint32_t smem_slot, uint32_t ncols) {

@@ -7,11 +7,12 @@
 //                          z    += row sums of the bf16 features (registers)
 //     softmax-token rows of the K / V tiles are copied from shared memory to the compact K_S / V_S.
 //   Q pass  (steps: softmax branch, phi_q projection, linear apply, merge)
-//     per 2 x 128 query rows: flash-style loop over 128-key tiles of K_S / V_S
-//                          S = Q K_S^T -> TMEM, running max / sum per row (one thread per row),
+//     persistent, one CTA per SM; per unit of 2 x 128 query rows a flash-style loop over 128-key tiles
+//     of K_S / V_S:        S = Q K_S^T -> TMEM, running max / sum per row (one thread per row),
 //                          P = exp2(.) as bf16 back into TMEM, O += P V_S (TMEM x smem)
-//     tail:                Phi = Q W_q^T -> TMEM, phi_q scaled per row -> smem, O += phi_q S,
-//                          den = l + phi_q.z, y = O / den -> bf16 -> TMA store.
+//     tail:                Phi = Q W_q^T -> TMEM (issued right behind the last P V), phi_q scaled per row
+//                          as bf16 where P sat, O += phi_q S (TMEM x smem, S in bf16 read like a V tile),
+//                          den = l + phi_q.z, y = O / den -> bf16 -> per-warp staging -> TMA store.
 // All tiles are staged by TMA with the 128-byte swizzle; every mbarrier wait is bounded.
 #include <cuda.h>
 
@@ -33,6 +34,7 @@ constexpr int BOX_BYTES = 128 * 128;     // one TMA box: 128 rows x 64 bf16 (128
 struct QParams {
   int N, n_s, nkv, lin, stab_mode, P, H;
   int layers;                // depth of the feature map: with 2, tmH holds relu(q W_1^T) and tmW is W_2
+  int nx, n_units;           // 256-row units per (batch, head); units over all (batch, head) pairs
   float scale_log2;          // softmax scale * log2(e)
   const float* z;            // [B*H][F]
   float* aux;                // [B*H][N][3] or nullptr
@@ -48,9 +50,10 @@ struct QLayout {
   static constexpr int TILE = 128 * D * 2;                 // bytes of a [128 x D] bf16 tile
   static constexpr int Q_OFF = 0;
   static constexpr int KV_OFF = 2 * TILE;
-  static constexpr int BAR_OFF = KV_OFF + KV_STAGES * TILE;
-  static constexpr int Z_OFF = BAR_OFF + 256;
-  static constexpr int TOTAL = Z_OFF + D * 4 + 1024;       // + slack for the 1024-byte alignment
+  static constexpr int OUT_OFF = KV_OFF + KV_STAGES * TILE;  // per softmax warp: 32 rows x 64 columns of bf16 output
+  static constexpr int OUT_WARP = 32 * 128;
+  static constexpr int BAR_OFF = OUT_OFF + 8 * OUT_WARP;
+  static constexpr int TOTAL = BAR_OFF + 256 + 1024;       // + slack for the 1024-byte alignment
 };
 
 // Loads a [128 x D] tile (rows y0.., of slice z) as D/64 swizzled boxes.
@@ -92,31 +95,388 @@ AS_DEV void store_row_chunk(uint8_t* tile, uint32_t row, uint32_t c0, const uint
   }
 }
 
+// Persistent: one CTA per SM walks over 256-row units (unit w = blockIdx.x + u * gridDim.x; the units of
+// one (batch, head) are consecutive, so the CTAs that run at the same time share K_S / V_S in L2).
+// Barrier phases and the K/V ring run on across units: the producer prefetches the next unit's first
+// key tiles and its Q tiles (as soon as the linear apply has released the Q buffer) while the softmax
+// warps still normalise and store the previous unit.
+//
+// The work of one unit is a function per role, kept out of line: each role then gets a register
+// allocation of its own (the softmax rows need nearly the whole budget, and the issuing thread must
+// not spill).  Everything about a unit is derived from its index u inside the function.
+struct QCtx {
+  uint32_t sbase;            // shared-memory window address of the 1024-aligned base
+  uint32_t tmem;             // TMEM base address
+  WaitCtx wc;
+};
+
+template <int D>
+struct QRing {
+  using L = QLayout<D>;
+  // barrier indices
+  static constexpr int B_Q0 = 0, B_FULL = 2, B_EMPTY = 2 + KV_STAGES, B_S = 2 + 2 * KV_STAGES, B_P = B_S + 2,
+                       B_O = B_P + 2, B_QF = B_O + 2, B_COUNT = B_QF + 2;
+  const QCtx c;              // by value: nothing here is re-read from memory after a barrier or an MMA
+  int it_w, it_h, it_st, n_items, n_sp;
+  // items of one unit: K and V tiles alternating, then for the linear tail the last-layer weights,
+  // (with a two-layer feature map) the two groups' first-layer activations, and S in bf16
+  AS_DEV QRing(int nkv, int lin, int layers, const QCtx& c_) : c(c_) {
+    it_w = 2 * nkv; it_h = 2 * nkv + 1; it_st = 2 * nkv + (layers == 2 ? 3 : 1);
+    n_items = lin ? it_st + 1 : 2 * nkv;
+    n_sp = nkv + lin;                    // completions of the S and of the P barrier per unit and group
+  }
+  AS_DEV uint32_t bar(int i) const { return c.sbase + L::BAR_OFF + 8 * i; }
+  AS_DEV uint32_t sQ(int g) const { return c.sbase + L::Q_OFF + g * L::TILE; }
+  // The K/V ring is indexed by a running item number that does not restart with a unit.
+  AS_DEV uint32_t sKV(int item) const { return c.sbase + L::KV_OFF + (item % KV_STAGES) * L::TILE; }
+  AS_DEV uint32_t tS(int g) const { return c.tmem + 128u * g; }
+  AS_DEV uint32_t tO(int g) const { return c.tmem + 256u + 128u * g; }
+  AS_DEV bool wait(int b, int phase) const { return mbar_wait_warp(bar(b), phase & 1, c.wc); }
+  AS_DEV bool full_wait(int item) const { return wait(B_FULL + item % KV_STAGES, item / KV_STAGES); }
+  AS_DEV void release(int item) const { tc_commit(bar(B_EMPTY + item % KV_STAGES)); }
+};
+
+// ---------------------------------------------------------------- TMA producer, one unit
+template <int D>
+__device__ __noinline__ bool q_produce_unit(const QParams& p, const QCtx& c, const CUtensorMap* tmQ, const CUtensorMap* tmK,
+                                            const CUtensorMap* tmV, const CUtensorMap* tmW, const CUtensorMap* tmSt,
+                                            const CUtensorMap* tmH, int u) {
+  using R = QRing<D>;
+  using L = QLayout<D>;
+  const int nkv = p.nkv;
+  const R q(nkv, p.lin, p.layers, c);
+  const int lane = threadIdx.x & 31;
+  const int w = (int)blockIdx.x + u * (int)gridDim.x;
+  const int bh = w / p.nx, h = bh % p.H, row0 = (w % p.nx) * 256;
+  const int base = u * q.n_items;
+  const int q_at = nkv > 0 ? 2 : 0;         // the Q tiles are requested after the unit's first K and V tile
+  for (int it = 0; it < q.n_items; ++it) {
+    if (it == q_at) {
+      for (int g = 0; g < 2; ++g) {
+        // the previous unit's last product that reads this Q buffer has completed
+        if (u > 0 && !q.wait(R::B_QF + g, u - 1)) return false;
+        if (lane == 0) {
+          mbar_expect_tx(q.bar(R::B_Q0 + g), L::TILE);
+          load_tile<D>(q.sQ(g), tmQ, q.bar(R::B_Q0 + g), row0 + g * 128, bh);
+        }
+        __syncwarp();
+      }
+    }
+    const int gi = base + it, st = gi % KV_STAGES;
+    if (!q.wait(R::B_EMPTY + st, gi / KV_STAGES + 1)) return false;
+    if (lane == 0) {
+      mbar_expect_tx(q.bar(R::B_FULL + st), L::TILE);
+      if (it < 2 * nkv) {
+        load_tile<D>(q.sKV(gi), (it & 1) ? tmV : tmK, q.bar(R::B_FULL + st), (it >> 1) * 128, bh);
+      } else if (it == q.it_w) {
+        load_tile<D>(q.sKV(gi), tmW, q.bar(R::B_FULL + st), 0, h);           // last-layer W_q[h]: [F rows][D]
+      } else if (it < q.it_st) {
+        load_tile<D>(q.sKV(gi), tmH, q.bar(R::B_FULL + st), row0 + (it - q.it_h) * 128, bh);   // relu(q W_1^T) of group it - it_h
+      } else {
+        load_tile<D>(q.sKV(gi), tmSt, q.bar(R::B_FULL + st), 0, bh);         // S[bh] in bf16: [F rows][D]
+      }
+    }
+    __syncwarp();
+  }
+  return true;
+}
+
+// ---------------------------------------------------------------- MMA issuer, one unit
+template <int D>
+__device__ __noinline__ bool q_mma_unit(const QParams& p, const QCtx& c, int u) {
+  using R = QRing<D>;
+  constexpr int F = D;
+  constexpr uint32_t ID_QK = make_idesc(128, 128, 0, 0);      // S = Q K^T      (N = 128 keys)
+  constexpr uint32_t ID_PV = make_idesc(128, D, 0, 1);        // O += P V and O += phi_q S  (V, S are MN-major)
+  constexpr uint32_t ID_PHI = make_idesc(128, F, 0, 0);       // Phi = Q W_q^T  (N = F)
+  const int nkv = p.nkv, lin = p.lin, layers = p.layers;
+  const R q(nkv, lin, layers, c);
+  const int lane = threadIdx.x & 31;
+  const int base = u * q.n_items, pb = u * q.n_sp;            // first ring item / first S,P phase of the unit
+  if (!q.wait(R::B_Q0, u)) return false;
+  if (nkv == 0 && !q.wait(R::B_Q0 + 1, u)) return false;
+  if (nkv > 0) {
+    if (!q.full_wait(base)) return false;
+    for (int g = 0; g < 2; ++g) {
+      if (g == 1 && !q.wait(R::B_Q0 + 1, u)) return false;
+      tc_fence_after();
+      if (lane == 0) {
+        issue_kmajor<D>(q.tS(g), kmajor_desc(q.sQ(g)), kmajor_desc(q.sKV(base)), ID_QK, false);
+        tc_commit(q.bar(R::B_S + g));
+        if (g == 1) q.release(base);
+      }
+      __syncwarp();
+    }
+    for (int j = 0; j < nkv; ++j) {
+      // this tile's V; the next tile's K, or after the last tile the feature weights: Phi = X W^T is
+      // issued right behind the group's last P V, in the place the next tile's Q K^T would have
+      const bool last = (j + 1 == nkv);
+      const int iv = base + 2 * j + 1, ik = last ? base + q.it_w : base + 2 * j + 2;
+      const uint32_t id_next = last ? ID_PHI : ID_QK;
+#pragma unroll
+      for (int g = 0; g < 2; ++g) {
+        // operands of the whole block are prepared before the wait, so that the issue itself is short
+        uint64_t dv[8], dq[8], dk[8];
+        uint32_t ap[8];
+        {
+          const uint32_t xa = (last && layers == 2) ? q.sKV(base + q.it_h + g) : q.sQ(g);
+          const uint64_t v0 = mnmajor_desc(q.sKV(iv)), q0 = kmajor_desc(xa), k0 = kmajor_desc(q.sKV(ik));
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint64_t off = (uint64_t)(((kk / 4) * BOX_BYTES + (kk % 4) * 32) >> 4);
+            dv[kk] = v0 + (uint64_t)((kk * 2048) >> 4);
+            dq[kk] = q0 + off;
+            dk[kk] = k0 + off;
+            ap[kk] = q.tS(g) + kk * 8;
+          }
+        }
+        if (!q.wait(R::B_P + g, pb + j)) return false;
+        if (g == 0 && !q.full_wait(iv)) return false;
+        if (g == 0 && (!last || lin) && !q.full_wait(ik)) return false;
+        if (last && layers == 2 && !q.full_wait(base + q.it_h + g)) return false;
+        tc_fence_after();
+        if (lane == 0) {
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) mma_ts(q.tO(g), ap[kk], dv[kk], ID_PV, (j > 0 || kk > 0) ? 1u : 0u);
+          if (!last || lin) {
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), dq[kk], dk[kk], id_next, kk > 0 ? 1u : 0u);
+            tc_commit(q.bar(R::B_S + g));
+          } else {
+            tc_commit(q.bar(R::B_O + g));
+          }
+          if (last) {
+            tc_commit(q.bar(R::B_QF + g));           // nothing of this unit reads the group's Q tile any more
+            if (layers == 2) q.release(base + q.it_h + g);
+          }
+        }
+        __syncwarp();
+      }
+      if (lane == 0) {
+        q.release(iv);
+        if (!last || lin) q.release(ik);
+      }
+      __syncwarp();
+    }
+  }
+  if (lin && nkv == 0) {
+    // no softmax tokens at all: the feature product opens the unit
+    if (!q.full_wait(base + q.it_w)) return false;
+    for (int g = 0; g < 2; ++g) {
+      // Phi = X W^T with X = Q (one layer) or the first-layer activations (two layers)
+      if (layers == 2 && !q.full_wait(base + q.it_h + g)) return false;
+      tc_fence_after();
+      if (lane == 0) {
+        issue_kmajor<D>(q.tS(g), kmajor_desc(layers == 2 ? q.sKV(base + q.it_h + g) : q.sQ(g)),
+                        kmajor_desc(q.sKV(base + q.it_w)), ID_PHI, false);
+        tc_commit(q.bar(R::B_S + g));
+        tc_commit(q.bar(R::B_QF + g));               // nothing of this unit reads the group's Q tile any more
+        if (layers == 2) q.release(base + q.it_h + g);
+        if (g == 1) q.release(base + q.it_w);
+      }
+      __syncwarp();
+    }
+  }
+  if (lin) {
+    if (!q.full_wait(base + q.it_st)) return false;
+    for (int g = 0; g < 2; ++g) {
+      if (!q.wait(R::B_P + g, pb + nkv)) return false;
+      tc_fence_after();
+      if (lane == 0) {
+        // phi_q sits where P sits (bf16 over the score columns), S plays the part of a V tile
+        const uint64_t s0 = mnmajor_desc(q.sKV(base + q.it_st));
+#pragma unroll
+        for (int kk = 0; kk < F / 16; ++kk)
+          mma_ts(q.tO(g), q.tS(g) + kk * 8, s0 + (uint64_t)((kk * 2048) >> 4), ID_PV, (nkv > 0 || kk > 0) ? 1u : 0u);
+        tc_commit(q.bar(R::B_O + g));
+        if (g == 1) q.release(base + q.it_st);
+      }
+      __syncwarp();
+    }
+  }
+  return true;
+}
+
+// ---------------------------------------------------------------- softmax / merge group, one unit
+template <int D>
+__device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, const CUtensorMap* tmO, uint8_t* smem, int u) {
+  using R = QRing<D>;
+  using L = QLayout<D>;
+  constexpr int F = D;
+  const int nkv = p.nkv, n_s = p.n_s;
+  const float scale_log2 = p.scale_log2;
+  const R q(nkv, p.lin, p.layers, c);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = warp >> 2;                          // group 0 or 1
+  const int r = (warp & 3) * 32 + lane;             // row inside the group's 128-row tile
+  const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+  const uint32_t tSg = q.tS(g) + lane_off, tOg = q.tO(g) + lane_off;
+  const int pb = u * q.n_sp;
+  float m_ref = 0.f, m_true = -INFINITY, l = 0.f;
+  uint32_t x[32];
+
+  for (int j = 0; j < nkv; ++j) {
+    if (!q.wait(R::B_S + g, pb + j)) return false;
+    tc_fence_after();
+    uint32_t sv[128];                               // this thread's row of the 128 x 128 score tile
+    tmem_ld128_sync(tSg, sv);
+    const int valid = n_s - j * 128;              // keys of this tile that exist (>= 128: all)
+    if (valid < 128) {
+#pragma unroll
+      for (int i = 0; i < 128; ++i) sv[i] = (i < valid) ? sv[i] : 0xff800000u;   // -inf: exp2 gives 0
+    }
+    float mx0 = fmax3(__uint_as_float(sv[0]), __uint_as_float(sv[1]), __uint_as_float(sv[2]));
+    float mx1 = fmax3(__uint_as_float(sv[3]), __uint_as_float(sv[4]), __uint_as_float(sv[5]));
+#pragma unroll
+    for (int i = 6; i + 3 < 128; i += 4) {
+      mx0 = fmax3(mx0, __uint_as_float(sv[i]), __uint_as_float(sv[i + 1]));
+      mx1 = fmax3(mx1, __uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3]));
+    }
+    float mx = fmax3(mx0, mx1, fmaxf(__uint_as_float(sv[126]), __uint_as_float(sv[127])));
+    mx *= scale_log2;
+    m_true = fmaxf(m_true, mx);
+    // The reference maximum only moves when the row maximum grew by more than 2^8; then O and l
+    // are rescaled (after P is out of the registers; the MMA that adds P V waits for this thread).
+    const bool need = (j > 0) && (mx > m_ref + RESCALE_THRESHOLD);
+    const float resc = need ? ex2(m_ref - mx) : 1.f;
+    if (j == 0 || need) m_ref = mx;
+    // P = exp2(s * scale_log2 - m_ref) as bf16, written over the first 64 columns of S
+    const float neg_m = -m_ref;
+    // packed fp32x2 arithmetic halves the instruction count of the scaling and of the row sum
+    const float2 scale2 = make_float2(scale_log2, scale_log2), negm2 = make_float2(neg_m, neg_m);
+    float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+      uint32_t pw[16];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int k = cc * 32 + 4 * i;
+        const float2 xa = __ffma2_rn(make_float2(__uint_as_float(sv[k]), __uint_as_float(sv[k + 1])), scale2, negm2);
+        const float2 xb = __ffma2_rn(make_float2(__uint_as_float(sv[k + 2]), __uint_as_float(sv[k + 3])), scale2, negm2);
+        const float2 pa = make_float2(ex2(xa.x), ex2(xa.y)), pc = make_float2(ex2(xb.x), ex2(xb.y));
+        la = __fadd2_rn(la, pa);
+        lb = __fadd2_rn(lb, pc);
+        pw[2 * i] = pack_bf16(pa.x, pa.y);
+        pw[2 * i + 1] = pack_bf16(pc.x, pc.y);
+      }
+      tmem_st16(tSg + cc * 16, pw);
+    }
+    l = l * resc + ((la.x + la.y) + (lb.x + lb.y));
+    if (__any_sync(0xffffffffu, need)) {
+      // O += P V of the previous tile has completed (its commit precedes this tile's S barrier)
+#pragma unroll
+      for (int cc = 0; cc < D / 32; ++cc) {
+        tmem_ld32(tOg + cc * 32, x);
+        tmem_ld_wait(x);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) x[i] = __float_as_uint(__uint_as_float(x[i]) * resc);
+        tmem_st32(tOg + cc * 32, x);
+      }
+    }
+    tmem_st_wait();
+    tc_fence_before();
+    mbar_arrive(q.bar(R::B_P + g));
+  }
+
+  const int w = (int)blockIdx.x + u * (int)gridDim.x;
+  const int bh = w / p.nx;
+  const int row = (w % p.nx) * 256 + g * 128 + r;
+  float den = l, den_l_out = 0.f;
+  if (p.lin) {
+    // per-row factor applied to phi_q so that the linear branch lands on the scale of O and l
+    float e = 0.f;
+    if (nkv > 0) e = (p.stab_mode == AS_STAB_EXACT) ? -m_ref : (m_true - m_ref);
+    e = fminf(fmaxf(e, -100.f), 100.f);
+    const float lam = ex2(e);
+    const float2* zrow = reinterpret_cast<const float2*>(p.z + (size_t)bh * F);
+    if (!q.wait(R::B_S + g, pb + nkv)) return false;
+    tc_fence_after();
+    float dl0 = 0.f, dl1 = 0.f;
+    const bool two_parts = (p.P == 2);
+#pragma unroll
+    for (int cc = 0; cc < F / 32; ++cc) {
+      tmem_ld32(tSg + cc * 32, x);
+      tmem_ld_wait(x);
+      const bool squared = two_parts && (cc * 32 >= F / 2);
+      uint32_t wd[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        float a0 = fmaxf(__uint_as_float(x[2 * i]), 0.f), a1 = fmaxf(__uint_as_float(x[2 * i + 1]), 0.f);
+        if (squared) { a0 *= a0; a1 *= a1; }
+        wd[i] = pack_bf16(a0 * lam, a1 * lam);
+        // the denominator uses the very bf16 values the MMA multiplies with S
+        const float2 zz = __ldg(zrow + cc * 16 + i);   // same address in every lane: one broadcast load
+        dl0 = fmaf(__uint_as_float(wd[i] << 16), zz.x, dl0);
+        dl1 = fmaf(__uint_as_float(wd[i] & 0xffff0000u), zz.y, dl1);
+      }
+      tmem_st16(tSg + cc * 16, wd);                  // over Phi columns this thread has already read
+    }
+    const float dl = dl0 + dl1;
+    tmem_st_wait();
+    tc_fence_before();
+    mbar_arrive(q.bar(R::B_P + g));
+    den = l + dl;
+    den_l_out = dl / lam;
+  }
+  if (!q.wait(R::B_O + g, u)) return false;
+  tc_fence_after();
+  const float inv = 1.f / den;
+  // Each warp stages its 32 rows, 64 columns at a time, in a buffer of its own and hands them to a
+  // TMA store (rows past N are clipped by the tensor map); no other warp is waited for.
+  uint8_t* stg = smem + L::OUT_OFF + warp * L::OUT_WARP;
+  const int wrow0 = row - lane;
+#pragma unroll
+  for (int half = 0; half < D / 64; ++half) {
+    uint32_t wd[32];
+#pragma unroll
+    for (int cc = 0; cc < 2; ++cc) {
+      tmem_ld32(tOg + half * 64 + cc * 32, x);
+      tmem_ld_wait(x);
+#pragma unroll
+      for (int i = 0; i < 16; ++i)
+        wd[cc * 16 + i] = pack_bf16(__uint_as_float(x[2 * i]) * inv, __uint_as_float(x[2 * i + 1]) * inv);
+    }
+    if (lane == 0) tma_store_wait_read();            // the buffer's previous store has been read out
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      *reinterpret_cast<uint4*>(stg + swz128_chunk_offset(lane, i)) =
+          make_uint4(wd[4 * i], wd[4 * i + 1], wd[4 * i + 2], wd[4 * i + 3]);
+    fence_proxy_async();
+    __syncwarp();
+    if (lane == 0 && wrow0 < p.N) {
+      tma_store_3d(tmO, smem_u32(stg), half * 64, wrow0, bh);
+      tma_store_commit();
+    }
+  }
+  if (p.aux != nullptr && row < p.N) {
+    const float ln2 = 0.6931471805599453f;
+    float* ap = p.aux + ((size_t)bh * p.N + row) * 3;
+    ap[0] = nkv > 0 ? m_true * ln2 : 0.f;
+    ap[1] = nkv > 0 ? l * ex2(m_ref - m_true) : 0.f;
+    ap[2] = den_l_out;
+  }
+  // The next unit's first P V overwrites O: every tcgen05.ld above has completed (tmem_ld_wait), and
+  // the arrive on the P barrier that releases that MMA follows in program order.
+  tc_fence_before();
+  return true;
+}
+
 template <int D>
 __global__ void __launch_bounds__(Q_THREADS, 1)
 qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
              const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmW,
-             const __grid_constant__ CUtensorMap tmSt, const __grid_constant__ CUtensorMap tmO,
-             const __grid_constant__ CUtensorMap tmH, const QParams p) {
+             const __grid_constant__ CUtensorMap tmSt, const __grid_constant__ CUtensorMap tmH,
+             const __grid_constant__ CUtensorMap tmO, const __grid_constant__ QParams p) {
   using L = QLayout<D>;
-  constexpr int F = D;
+  using R = QRing<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::BAR_OFF);
-  // barrier indices
-  enum { B_Q0 = 0, B_FULL = 2, B_EMPTY = 2 + KV_STAGES, B_S = 2 + 2 * KV_STAGES, B_P = B_S + 2, B_O = B_P + 2,
-         B_COUNT = B_O + 2 };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::BAR_OFF + 8 * B_COUNT);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::BAR_OFF + 8 * B_COUNT + 4);
-  float* sZ = reinterpret_cast<float*>(smem + L::Z_OFF);
-  auto bar = [&](int i) { return smem_u32(bars + i); };
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int bh = blockIdx.y, h = bh % p.H;
-  const int row0 = blockIdx.x * 256;
-  const int nkv = p.nkv;
-  const WaitCtx wc{p.status, abort_flag};
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::BAR_OFF + 8 * R::B_COUNT);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::BAR_OFF + 8 * R::B_COUNT + 4);
+  auto bar = [&](int i) { return sbase + L::BAR_OFF + 8 * i; };
+  const int warp = threadIdx.x >> 5;
 
   // an earlier CTA of this or a previous launch timed out: do nothing (decided once per CTA)
   __shared__ uint32_t s_skip;
@@ -126,280 +486,32 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 
   if (threadIdx.x == 0) {
     *abort_flag = 0u;
-    mbar_init(bar(B_Q0), 1); mbar_init(bar(B_Q0 + 1), 1);
-    for (int s = 0; s < KV_STAGES; ++s) { mbar_init(bar(B_FULL + s), 1); mbar_init(bar(B_EMPTY + s), 1); }
-    for (int g = 0; g < 2; ++g) { mbar_init(bar(B_S + g), 1); mbar_init(bar(B_P + g), 128); mbar_init(bar(B_O + g), 1); }
+    mbar_init(bar(R::B_Q0), 1); mbar_init(bar(R::B_Q0 + 1), 1);
+    for (int s = 0; s < KV_STAGES; ++s) { mbar_init(bar(R::B_FULL + s), 1); mbar_init(bar(R::B_EMPTY + s), 1); }
+    for (int g = 0; g < 2; ++g) {
+      mbar_init(bar(R::B_S + g), 1); mbar_init(bar(R::B_P + g), 128); mbar_init(bar(R::B_O + g), 1); mbar_init(bar(R::B_QF + g), 1);
+    }
     fence_barrier_init();
     fence_proxy_async();
   }
-  if (p.lin && threadIdx.x < F) sZ[threadIdx.x] = p.z[(size_t)bh * F + threadIdx.x];
   if (warp == 9) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
-  const uint32_t tS[2] = {tmem + 0u, tmem + 128u};
-  const uint32_t tO[2] = {tmem + 256u, tmem + 384u};
-  const uint32_t sQ[2] = {sbase + L::Q_OFF, sbase + L::Q_OFF + L::TILE};
-  auto sKV = [&](int item) { return sbase + L::KV_OFF + (item % KV_STAGES) * L::TILE; };
-  // items of the K/V ring: K and V tiles alternating, then for the linear tail the last-layer weights,
-  // (with a two-layer feature map) the two groups' first-layer activations, and S^T
-  const int it_w = 2 * nkv, it_h = 2 * nkv + 1, it_st = 2 * nkv + (p.layers == 2 ? 3 : 1);
-  const int n_items = p.lin ? it_st + 1 : 2 * nkv;
+  const QCtx c{sbase, *tmem_slot, WaitCtx{p.status, abort_flag}};
+  const int n_mine = (p.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // units of this CTA
 
   if (warp == 8) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmO);
-      for (int g = 0; g < 2; ++g) {
-        mbar_expect_tx(bar(B_Q0 + g), L::TILE);
-        load_tile<D>(sQ[g], &tmQ, bar(B_Q0 + g), row0 + g * 128, bh);
-      }
-    }
-    for (int it = 0; it < n_items; ++it) {
-      const int st = it % KV_STAGES, use = it / KV_STAGES;
-      if (!mbar_wait_warp(bar(B_EMPTY + st), (use & 1) ^ 1, wc)) break;
-      if (lane == 0) {
-        mbar_expect_tx(bar(B_FULL + st), L::TILE);
-        if (it < 2 * nkv) {
-          const int j = it >> 1;
-          load_tile<D>(sKV(it), (it & 1) ? &tmV : &tmK, bar(B_FULL + st), j * 128, bh);
-        } else if (it == it_w) {
-          load_tile<D>(sKV(it), &tmW, bar(B_FULL + st), 0, h);          // W_q[h]: [F rows][D]
-        } else if (it < it_st) {
-          load_tile<D>(sKV(it), &tmH, bar(B_FULL + st), row0 + (it - it_h) * 128, bh);   // relu(q W_1^T) of group it - it_h
-        } else {
-          load_tile<D>(sKV(it), &tmSt, bar(B_FULL + st), 0, bh);        // S^T[bh]: [D rows][F]
-        }
-      }
-      __syncwarp();
-    }
+    if ((threadIdx.x & 31) == 0) { tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmO); }
+    for (int u = 0; u < n_mine; ++u)
+      if (!q_produce_unit<D>(p, c, &tmQ, &tmK, &tmV, &tmW, &tmSt, &tmH, u)) break;
   } else if (warp == 9) {
-    // ------------------------------------------------------------ MMA issuer
-    constexpr uint32_t ID_QK = make_idesc(128, 128, 0, 0);      // S = Q K^T      (N = 128 keys)
-    constexpr uint32_t ID_PV = make_idesc(128, D, 0, 1);        // O += P V       (V is MN-major)
-    constexpr uint32_t ID_PHI = make_idesc(128, F, 0, 0);       // Phi = Q W_q^T  (N = F)
-    constexpr uint32_t ID_LIN = make_idesc(128, D, 0, 0);       // O += phi_q S   (B = S^T, K-major)
-    auto full_wait = [&](int item) { return mbar_wait_warp(bar(B_FULL + item % KV_STAGES), (item / KV_STAGES) & 1, wc); };
-    bool ok = mbar_wait_warp(bar(B_Q0), 0, wc) && mbar_wait_warp(bar(B_Q0 + 1), 0, wc);
-    if (ok && nkv > 0) {
-      ok = full_wait(0);
-      if (ok) {
-        tc_fence_after();
-        if (lane == 0) {
-          for (int g = 0; g < 2; ++g) { issue_kmajor<D>(tS[g], kmajor_desc(sQ[g]), kmajor_desc(sKV(0)), ID_QK, false); tc_commit(bar(B_S + g)); }
-          tc_commit(bar(B_EMPTY + 0));
-        }
-        __syncwarp();
-      }
-      for (int j = 0; ok && j < nkv; ++j) {
-#pragma unroll
-        for (int g = 0; g < 2; ++g) {
-          if (!ok) break;
-          // operands of the whole block are prepared before the wait, so that the issue itself is short
-          uint64_t dv[8], dq[8], dk[8];
-          uint32_t ap[8];
-          {
-            const uint64_t v0 = mnmajor_desc(sKV(2 * j + 1)), q0 = kmajor_desc(sQ[g]), k0 = kmajor_desc(sKV(2 * j + 2));
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-              const uint64_t off = (uint64_t)(((kk / 4) * BOX_BYTES + (kk % 4) * 32) >> 4);
-              dv[kk] = v0 + (uint64_t)((kk * 2048) >> 4);
-              dq[kk] = q0 + off;
-              dk[kk] = k0 + off;
-              ap[kk] = tS[g] + kk * 8;
-            }
-          }
-          ok = mbar_wait_warp(bar(B_P + g), j & 1, wc);
-          if (ok && g == 0) ok = full_wait(2 * j + 1);
-          if (ok && g == 0 && j + 1 < nkv) ok = full_wait(2 * j + 2);
-          if (!ok) break;
-          tc_fence_after();
-          if (lane == 0) {
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) mma_ts(tO[g], ap[kk], dv[kk], ID_PV, (j > 0 || kk > 0) ? 1u : 0u);
-            if (j + 1 < nkv) {
-#pragma unroll
-              for (int kk = 0; kk < D / 16; ++kk) mma_ss(tS[g], dq[kk], dk[kk], ID_QK, kk > 0 ? 1u : 0u);
-              tc_commit(bar(B_S + g));
-            } else if (!p.lin) {
-              tc_commit(bar(B_O + g));
-            }
-          }
-          __syncwarp();
-        }
-        if (ok && lane == 0) {
-          tc_commit(bar(B_EMPTY + (2 * j + 1) % KV_STAGES));
-          if (j + 1 < nkv) tc_commit(bar(B_EMPTY + (2 * j + 2) % KV_STAGES));
-        }
-        __syncwarp();
-      }
-    }
-    if (ok && p.lin) {
-      ok = full_wait(it_w);
-      for (int g = 0; ok && g < 2; ++g) {
-        // Phi = X W^T with X = Q (one layer) or the first-layer activations (two layers)
-        if (p.layers == 2) ok = full_wait(it_h + g);
-        if (!ok) break;
-        tc_fence_after();
-        if (lane == 0) {
-          issue_kmajor<D>(tS[g], kmajor_desc(p.layers == 2 ? sKV(it_h + g) : sQ[g]), kmajor_desc(sKV(it_w)), ID_PHI, false);
-          tc_commit(bar(B_S + g));
-        }
-        __syncwarp();
-      }
-      if (ok) ok = full_wait(it_st);
-      for (int g = 0; ok && g < 2; ++g) {
-        ok = mbar_wait_warp(bar(B_P + g), nkv & 1, wc);
-        if (!ok) break;
-        tc_fence_after();
-        if (lane == 0) {
-          issue_kmajor<F>(tO[g], kmajor_desc(sQ[g]), kmajor_desc(sKV(it_st)), ID_LIN, nkv > 0);
-          tc_commit(bar(B_O + g));
-        }
-        __syncwarp();
-      }
-    }
+    for (int u = 0; u < n_mine; ++u)
+      if (!q_mma_unit<D>(p, c, u)) break;
   } else {
-    // ------------------------------------------------------------ softmax / merge groups
-    const int g = warp >> 2;                          // group 0 or 1
-    const int r = (warp & 3) * 32 + lane;             // row inside the group's 128-row tile
-    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tSg = tS[g] + lane_off, tOg = tO[g] + lane_off;
-    const int row = row0 + g * 128 + r;
-    uint8_t* sQg = smem + L::Q_OFF + g * L::TILE;
-    float m_ref = 0.f, m_true = -INFINITY, l = 0.f;
-    bool ok = true;
-    uint32_t x[32];
-
-    for (int j = 0; j < nkv; ++j) {
-      ok = mbar_wait_warp(bar(B_S + g), j & 1, wc);
-      if (!ok) break;
-      tc_fence_after();
-      uint32_t sv[128];                               // this thread's row of the 128 x 128 score tile
-      tmem_ld128_sync(tSg, sv);
-      const int valid = p.n_s - j * 128;              // keys of this tile that exist (>= 128: all)
-      if (valid < 128) {
-#pragma unroll
-        for (int i = 0; i < 128; ++i) sv[i] = (i < valid) ? sv[i] : 0xff800000u;   // -inf: exp2 gives 0
-      }
-      float mx0 = fmax3(__uint_as_float(sv[0]), __uint_as_float(sv[1]), __uint_as_float(sv[2]));
-      float mx1 = fmax3(__uint_as_float(sv[3]), __uint_as_float(sv[4]), __uint_as_float(sv[5]));
-#pragma unroll
-      for (int i = 6; i + 3 < 128; i += 4) {
-        mx0 = fmax3(mx0, __uint_as_float(sv[i]), __uint_as_float(sv[i + 1]));
-        mx1 = fmax3(mx1, __uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3]));
-      }
-      float mx = fmax3(mx0, mx1, fmaxf(__uint_as_float(sv[126]), __uint_as_float(sv[127])));
-      mx *= p.scale_log2;
-      m_true = fmaxf(m_true, mx);
-      // The reference maximum only moves when the row maximum grew by more than 2^8; then O and l
-      // are rescaled (after P is out of the registers; the MMA that adds P V waits for this thread).
-      const bool need = (j > 0) && (mx > m_ref + RESCALE_THRESHOLD);
-      const float resc = need ? ex2(m_ref - mx) : 1.f;
-      if (j == 0 || need) m_ref = mx;
-      // P = exp2(s * scale_log2 - m_ref) as bf16, written over the first 64 columns of S
-      const float neg_m = -m_ref;
-      // packed fp32x2 arithmetic halves the instruction count of the scaling and of the row sum
-      const float2 scale2 = make_float2(p.scale_log2, p.scale_log2), negm2 = make_float2(neg_m, neg_m);
-      float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t pw[16];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int k = c * 32 + 4 * i;
-          const float2 xa = __ffma2_rn(make_float2(__uint_as_float(sv[k]), __uint_as_float(sv[k + 1])), scale2, negm2);
-          const float2 xb = __ffma2_rn(make_float2(__uint_as_float(sv[k + 2]), __uint_as_float(sv[k + 3])), scale2, negm2);
-          const float2 pa = make_float2(ex2(xa.x), ex2(xa.y)), pb = make_float2(ex2(xb.x), ex2(xb.y));
-          la = __fadd2_rn(la, pa);
-          lb = __fadd2_rn(lb, pb);
-          pw[2 * i] = pack_bf16(pa.x, pa.y);
-          pw[2 * i + 1] = pack_bf16(pb.x, pb.y);
-        }
-        tmem_st16(tSg + c * 16, pw);
-      }
-      l = l * resc + ((la.x + la.y) + (lb.x + lb.y));
-      if (__any_sync(0xffffffffu, need)) {
-        // O += P V of the previous tile has completed (its commit precedes this tile's S barrier)
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          tmem_ld32(tOg + c * 32, x);
-          tmem_ld_wait(x);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) x[i] = __float_as_uint(__uint_as_float(x[i]) * resc);
-          tmem_st32(tOg + c * 32, x);
-        }
-      }
-      tmem_st_wait();
-      tc_fence_before();
-      mbar_arrive(bar(B_P + g));
-    }
-
-    float den = l, den_l_out = 0.f;
-    if (ok && p.lin) {
-      // per-row factor applied to phi_q so that the linear branch lands on the scale of O and l
-      float e = 0.f;
-      if (nkv > 0) e = (p.stab_mode == AS_STAB_EXACT) ? -m_ref : (m_true - m_ref);
-      e = fminf(fmaxf(e, -100.f), 100.f);
-      const float lam = ex2(e);
-      ok = mbar_wait_warp(bar(B_S + g), nkv & 1, wc);
-      if (ok) {
-        tc_fence_after();
-        float dl = 0.f;
-#pragma unroll
-        for (int c = 0; c < F / 32; ++c) {
-          tmem_ld32(tSg + c * 32, x);
-          tmem_ld_wait(x);
-          const bool squared = (p.P == 2) && (c * 32 >= F / 2);
-          uint32_t w[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float a0 = fmaxf(__uint_as_float(x[2 * i]), 0.f), a1 = fmaxf(__uint_as_float(x[2 * i + 1]), 0.f);
-            if (squared) { a0 *= a0; a1 *= a1; }
-            a0 = bf16_round(a0 * lam); a1 = bf16_round(a1 * lam);
-            dl = fmaf(a0, sZ[c * 32 + 2 * i], dl);
-            dl = fmaf(a1, sZ[c * 32 + 2 * i + 1], dl);
-            w[i] = pack_bf16(a0, a1);
-          }
-          store_row_chunk(sQg, r, c * 32, w);        // Q itself is no longer needed: Phi has completed
-        }
-        fence_proxy_async();
-        mbar_arrive(bar(B_P + g));
-        den = l + dl;
-        den_l_out = dl / lam;
-      }
-    }
-    if (ok) ok = mbar_wait_warp(bar(B_O + g), 0, wc);
-    if (ok) {
-      tc_fence_after();
-      const float inv = 1.f / den;
-#pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        tmem_ld32(tOg + c * 32, x);
-        tmem_ld_wait(x);
-        uint32_t w[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-          w[i] = pack_bf16(__uint_as_float(x[2 * i]) * inv, __uint_as_float(x[2 * i + 1]) * inv);
-        store_row_chunk(sQg, r, c * 32, w);
-      }
-      fence_proxy_async();
-      named_barrier_sync(1 + g, 128);
-      if (r == 0 && row0 + g * 128 < p.N) {
-#pragma unroll
-        for (int b = 0; b < D / 64; ++b) tma_store_3d(&tmO, smem_u32(sQg) + b * BOX_BYTES, b * 64, row0 + g * 128, bh);
-        tma_store_commit();
-        tma_store_wait_all();
-      }
-      if (p.aux != nullptr && row < p.N) {
-        const float ln2 = 0.6931471805599453f;
-        float* ap = p.aux + ((size_t)bh * p.N + row) * 3;
-        ap[0] = nkv > 0 ? m_true * ln2 : 0.f;
-        ap[1] = nkv > 0 ? l * ex2(m_ref - m_true) : 0.f;
-        ap[2] = den_l_out;
-      }
-    }
+    for (int u = 0; u < n_mine; ++u)
+      if (!q_softmax_unit<D>(p, c, &tmO, smem, u)) break;
+    if ((threadIdx.x & 31) == 0) tma_store_wait_all();   // this warp's output stores have completed
   }
 
   // ------------------------------------------------------------ teardown
@@ -407,7 +519,7 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   __syncthreads();
   if (warp == 9) {
     tc_fence_after();
-    tmem_dealloc(tmem, 512);
+    tmem_dealloc(c.tmem, 512);
   }
 }
 
@@ -862,8 +974,9 @@ cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st) {
   if (g_encode == nullptr) return cudaErrorNotSupported;
   const int BH = a.B * a.H;
   const bool lin = a.n_l > 0;
-  CUtensorMap tmQ, tmK, tmV, tmW, tmSt, tmO, tmH;
-  if (!make_map(&tmQ, a.q, a.d, a.N, BH, 128) || !make_map(&tmO, a.out, a.d, a.N, BH, 128)) return cudaErrorInvalidValue;
+  CUtensorMap tmQ, tmK, tmV, tmW, tmSt, tmH, tmO;
+  // the output is stored warp by warp: boxes of 32 rows
+  if (!make_map(&tmQ, a.q, a.d, a.N, BH, 128) || !make_map(&tmO, a.out, a.d, a.N, BH, 32)) return cudaErrorInvalidValue;
   if (a.n_s > 0) {
     if (!make_map(&tmK, a.ks, a.d, a.n_s, BH, 128) || !make_map(&tmV, a.vs, a.d, a.n_s, BH, 128)) return cudaErrorInvalidValue;
   } else {
@@ -871,7 +984,7 @@ cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st) {
   }
   if (lin) {
     // boxes are always 128 rows: rows past F (or d) are out of bounds and arrive as zeros
-    if (!make_map(&tmW, a.layers == 2 ? a.wq2 : a.wq, a.d, a.F, a.H, 128) || !make_map(&tmSt, a.St, a.F, a.d, BH, 128)) return cudaErrorInvalidValue;
+    if (!make_map(&tmW, a.layers == 2 ? a.wq2 : a.wq, a.d, a.F, a.H, 128) || !make_map(&tmSt, a.Sb, a.d, a.F, BH, 128)) return cudaErrorInvalidValue;
   } else {
     tmW = tmQ; tmSt = tmQ;      // never used: no linear branch at rate 1
   }
@@ -883,8 +996,14 @@ cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st) {
   p.H = a.H;
   p.scale_log2 = a.scale * 1.4426950408889634f;
   p.z = a.z; p.aux = a.aux; p.status = a.status;
-  dim3 grid((a.N + 255) / 256, BH, 1);
-  if (a.d == 128) qpass_kernel<128><<<grid, Q_THREADS, QLayout<128>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmO, tmH, p);
-  else qpass_kernel<64><<<grid, Q_THREADS, QLayout<64>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmO, tmH, p);
+  p.nx = (a.N + 255) / 256;
+  p.n_units = p.nx * BH;
+  // persistent: one CTA per SM (the kernel's shared memory and its 512 TMEM columns allow no second one)
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+    return cudaErrorInvalidValue;
+  dim3 grid(p.n_units < sms ? p.n_units : sms, 1, 1);
+  if (a.d == 128) qpass_kernel<128><<<grid, Q_THREADS, QLayout<128>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmH, tmO, p);
+  else qpass_kernel<64><<<grid, Q_THREADS, QLayout<64>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmH, tmO, p);
   return cudaGetLastError();
 }
