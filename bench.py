@@ -309,7 +309,9 @@ def run_ours(args, wl):
                     "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                     "traffic": QPASS_DRAM_TRAFFIC_BYTES.get(wl.name),
                     "peak_source": "%s burst bf16 (sustained %s)" % (peaks["source"], peaks["bf16_tflops_sustained"]),
-                    "frac_of_nominal_2250": achieved / 2250.0, "avg_launch_ms": q_ms,
+                    "frac_of_nominal_2250": achieved / 2250.0,
+                    "frac_of_sustained": (achieved / peaks["bf16_tflops_sustained"]) if peaks.get("bf16_tflops_sustained") else None,
+                    "avg_launch_ms": q_ms,
                     "flops_per_launch": fl["qpass"]}
         else:       # rate 0: the whole layer is bound by reading q, k, v and writing out
             gbs = bytes_per_layer(wl) / ((k_ms + r_ms + q_ms) * 1e-3) / 1e9
