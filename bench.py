@@ -388,9 +388,18 @@ def run_stack(args):
         del op, dev, out
     total = sum(v["ms_per_layer"] * v["layers"] for v in per_rate.values())
     all_softmax = per_rate[1]["ms_per_layer"] * len(sched)
+    # Block-rate selection with the costs just measured and synthetic per-block errors: the same budget
+    # as the fixed schedule, spent where the (synthetic) error falls fastest.
+    from paper_2509_24899_b200 import binding
+    err = W.stack_errors(0)
+    cost = [[per_rate[r]["ms_per_layer"] for r in W.STACK_RATES] for _ in sched]
+    choice, sel_ms, sel_err = binding.as_select_block_rates(cost, err.tolist(), total)
+    fixed_err = float(sum(err[i][W.STACK_RATES.index(r)] for i, r in enumerate(sched)))
+    selection = {"budget_ms": total, "selected_ms": sel_ms, "selected_err": sel_err, "fixed_schedule_err": fixed_err,
+                 "selected_rates": [W.STACK_RATES[c] for c in choice], "errors": "synthetic"}
     print(json.dumps({"workload": "stack", "schedule": sched, "per_rate": {str(k): v for k, v in per_rate.items()},
                       "stack_ms": total, "all_softmax_ms": all_softmax, "speedup_vs_all_softmax": all_softmax / total,
-                      "dtype": "bf16", "data": "synthetic"}))
+                      "block_rate_selection": selection, "dtype": "bf16", "data": "synthetic"}))
     return 0
 
 

@@ -52,7 +52,8 @@ typedef enum {
   AS_ERR_ALLOC = 4,           /* host or device allocation failed in create                        */
   AS_ERR_WORKSPACE = 5,       /* workspace NULL, misaligned or smaller than workspace_bytes         */
   AS_ERR_CUDA = 6,            /* a CUDA runtime/driver call failed                                  */
-  AS_ERR_DEVICE_TIMEOUT = 7   /* a bounded wait inside a kernel ran out (see last_status)           */
+  AS_ERR_DEVICE_TIMEOUT = 7,  /* a bounded wait inside a kernel ran out (see last_status)           */
+  AS_ERR_INFEASIBLE = 8       /* block-rate selection: no assignment fits the budget                */
 } as_status_t;
 
 /* Stabiliser handling (the paper subtracts c_i only inside the softmax exponentials):
@@ -191,6 +192,25 @@ AS_API as_status_t as_hybrid_attn_linear_state_static(
     const void* k, const void* v, const void* wk, int32_t B, int32_t H, int32_t N, int32_t d,
     int32_t grid_t, int32_t grid_h, int32_t grid_w, int32_t blk_t, int32_t blk_h, int32_t blk_w,
     int32_t rate_den, int32_t poly_degree, float* S_out, float* z_out, void* cuda_stream);
+
+/* Block-rate selection (paragraph "Heterogeneous Block-Rate Optimization"): with n_blocks
+ * transformer blocks and n_rates candidate hybrid rates, pick one rate per block so that the summed
+ * error is minimal while the summed cost stays within `budget` (a multiple-choice knapsack problem).
+ *   cost, err  [n_blocks, n_rates] float64, HOST, row-major, read only: c_ir (FLOPs, latency, ... any
+ *              non-negative unit, e.g. per-layer times measured with this library) and e_ir (error
+ *              of block i at rate r relative to softmax attention); all finite
+ *   budget     beta, in the unit of `cost`; a summed cost equal to it is allowed
+ *   choice_out [n_blocks] int32, HOST, written: the chosen rate index per block
+ *   total_cost_out, total_err_out   HOST, written when not NULL: the sums over the chosen entries,
+ *              added in block order
+ * Exact (no cost discretisation): non-dominated partial assignments are carried from block to block.
+ * Where several assignments reach the minimal error, one of them is returned.  Host code only; no
+ * CUDA call, no stream.  Errors: AS_ERR_INVALID_ARG (NULL, non-positive sizes, NaN/inf or negative
+ * cost), AS_ERR_INFEASIBLE (even the cheapest rates exceed the budget; outputs untouched),
+ * AS_ERR_UNSUPPORTED (more than 2^22 non-dominated partial assignments), AS_ERR_ALLOC. */
+AS_API as_status_t as_select_block_rates(int32_t n_blocks, int32_t n_rates, const double* cost, const double* err,
+                                         double budget, int32_t* choice_out, double* total_cost_out,
+                                         double* total_err_out);
 
 /* Static description of a status code. */
 AS_API const char* as_status_string(as_status_t s);

@@ -7,9 +7,10 @@ from __future__ import annotations
 
 from . import binding
 from .binding import (AS_PATH_SIMT, AS_PATH_TENSOR, AS_STAB_EXACT, AS_STAB_PAPER, AsError)
+from .binding import as_select_block_rates as select_block_rates
 
 __all__ = ["binding", "HybridAttention", "AS_PATH_SIMT", "AS_PATH_TENSOR", "AS_STAB_EXACT",
-           "AS_STAB_PAPER", "AsError"]
+           "AS_STAB_PAPER", "AsError", "select_block_rates"]
 
 
 class HybridAttention:

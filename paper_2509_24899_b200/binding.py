@@ -13,7 +13,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "lib", "libas_hybrid_attn.so")
 
 AS_OK, AS_ERR_INVALID_ARG, AS_ERR_UNSUPPORTED, AS_ERR_ARCH = 0, 1, 2, 3
-AS_ERR_ALLOC, AS_ERR_WORKSPACE, AS_ERR_CUDA, AS_ERR_DEVICE_TIMEOUT = 4, 5, 6, 7
+AS_ERR_ALLOC, AS_ERR_WORKSPACE, AS_ERR_CUDA, AS_ERR_DEVICE_TIMEOUT, AS_ERR_INFEASIBLE = 4, 5, 6, 7, 8
 AS_STAB_PAPER, AS_STAB_EXACT = 0, 1
 AS_ACT_RELU = 0
 AS_PATH_TENSOR, AS_PATH_SIMT = 0, 1
@@ -76,6 +76,8 @@ def lib() -> C.CDLL:
             "as_hybrid_attn_launch_count": [H, C.POINTER(C.c_uint64)],
             "as_hybrid_attn_linear_state_static": [C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 12
                                                   + [C.c_void_p, C.c_void_p, C.c_void_p],
+            "as_select_block_rates": [C.c_int32, C.c_int32, C.POINTER(C.c_double), C.POINTER(C.c_double), C.c_double,
+                                      C.POINTER(C.c_int32), C.POINTER(C.c_double), C.POINTER(C.c_double)],
         }
         for name, args in sigs.items():
             fn = getattr(L, name)
@@ -214,3 +216,23 @@ def as_hybrid_attn_linear_state_static(k_ptr, v_ptr, wk_ptr, B, H, N, d, grid, b
     _check(lib().as_hybrid_attn_linear_state_static(
         k_ptr, v_ptr, wk_ptr, B, H, N, d, grid[0], grid[1], grid[2], block[0], block[1], block[2], rate,
         poly_degree, S_ptr or None, z_ptr or None, stream_ptr or None), "as_hybrid_attn_linear_state_static")
+
+
+def as_select_block_rates(cost, err, budget):
+    """One rate index per block with minimal summed error under the cost budget.
+
+    cost, err: [n_blocks][n_rates] (anything convertible to rows of floats).  Returns
+    (choice: list of int, total_cost, total_err); raises AsError(AS_ERR_INFEASIBLE) when even the
+    cheapest rates exceed the budget.  Host computation inside the library; no GPU is needed."""
+    n_blocks = len(cost)
+    n_rates = len(cost[0]) if n_blocks else 0
+    if n_blocks == 0 or n_rates == 0 or len(err) != n_blocks or any(len(r) != n_rates for r in cost) \
+            or any(len(r) != n_rates for r in err):
+        raise AsError(AS_ERR_INVALID_ARG, "as_select_block_rates")
+    flat_c = (C.c_double * (n_blocks * n_rates))(*[float(x) for row in cost for x in row])
+    flat_e = (C.c_double * (n_blocks * n_rates))(*[float(x) for row in err for x in row])
+    choice = (C.c_int32 * n_blocks)()
+    tc, te = C.c_double(), C.c_double()
+    _check(lib().as_select_block_rates(n_blocks, n_rates, flat_c, flat_e, float(budget), choice,
+                                       C.byref(tc), C.byref(te)), "as_select_block_rates")
+    return list(choice), tc.value, te.value

@@ -113,6 +113,7 @@ const char* as_status_string(as_status_t s) {
     case AS_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case AS_ERR_CUDA: return "CUDA call failed";
     case AS_ERR_DEVICE_TIMEOUT: return "bounded wait inside a kernel expired";
+    case AS_ERR_INFEASIBLE: return "no assignment fits the budget";
   }
   return "unknown status";
 }

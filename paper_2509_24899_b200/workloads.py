@@ -79,6 +79,16 @@ def stack_schedule(seed: int = 0, layers: int = STACK_LAYERS):
     return [STACK_RATES[next(gen) % len(STACK_RATES)] for _ in range(layers)]
 
 
+def stack_errors(seed: int = 0, layers: int = STACK_LAYERS) -> np.ndarray:
+    """Synthetic per-block errors e_ir [layers][len(STACK_RATES)] for the block-rate selection: zero at
+    rate 1, growing towards sparser rates, with a per-block sensitivity spread over a decade (stand-ins
+    for the distillation errors, which need the trained model)."""
+    rng = np.random.default_rng(9000 + seed)
+    steps = rng.uniform(0.2, 1.0, (layers, len(STACK_RATES)))
+    steps[:, 0] = 0.0
+    return np.cumsum(steps, axis=1) * np.exp(rng.uniform(np.log(0.3), np.log(3.0), (layers, 1)))
+
+
 def stack_layer(layer: int, seed: int = 0) -> Workload:
     """Workload of one layer of the 30-layer stack (headline shape, scheduled rate)."""
     rate = stack_schedule(seed)[layer]
