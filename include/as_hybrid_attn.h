@@ -133,9 +133,12 @@ AS_API as_status_t as_hybrid_attn_forward(as_hybrid_attn_t h, const void* q, con
                                    const as_phi_weights_t* w, void* out, float* aux,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* Same operation with HOST q, k, v and out buffers (pinned memory keeps the copies asynchronous):
- * copies q, k, v to staging space in the workspace, runs forward, copies the result back, all on
- * the stream.  The weights stay device pointers.  workspace >= workspace_bytes_host. */
+/* Same operation with HOST q, k, v and out buffers (pinned memory keeps the copies asynchronous).
+ * The work is cut into runs of whole heads (about 8 MB of q or more each): the copies in of one run,
+ * the kernels of the previous one and the copy out of the one before overlap, on two side streams the
+ * handle creates on the first call.  Everything is ordered after the work already in `cuda_stream`,
+ * and `cuda_stream` completes only after the last copy out.  The weights stay device pointers.
+ * workspace >= workspace_bytes_host.  Not for use by two host threads on one handle at once. */
 AS_API as_status_t as_hybrid_attn_forward_host(as_hybrid_attn_t h, const void* q_host, const void* k_host,
                                         const void* v_host, const as_phi_weights_t* w,
                                         void* out_host, void* workspace, size_t workspace_bytes,

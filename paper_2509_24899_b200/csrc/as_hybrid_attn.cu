@@ -101,6 +101,22 @@ struct ProfileScope {
 
 }  // namespace
 
+static as_status_t launch_heads(as_hybrid_attn_t h, const void* q, const void* k, const void* v,
+                                const as_phi_weights_t* w, void* out, float* aux, char* ws, cudaStream_t st,
+                                int first, int count, int nb, int nh);
+
+// The feature-map weights a layer with linear tokens needs: present, 16-byte aligned, no biases.
+static as_status_t check_weights(const as_hybrid_attn_s* h, const as_phi_weights_t* w) {
+  if (h->n_l == 0) return AS_OK;
+  const auto& d = h->desc;
+  if (!w || !w->wq1 || !w->wk1) return AS_ERR_INVALID_ARG;
+  if (w->bq1 || w->bk1 || w->bq2 || w->bk2) return AS_ERR_UNSUPPORTED;
+  if (d.phi_layers == 1 && (w->wq2 || w->wk2)) return AS_ERR_INVALID_ARG;
+  if (d.phi_layers == 2 && (!w->wq2 || !w->wk2)) return AS_ERR_INVALID_ARG;
+  if (((uintptr_t)w->wq1 | (uintptr_t)w->wk1 | (uintptr_t)w->wq2 | (uintptr_t)w->wk2) & 15) return AS_ERR_INVALID_ARG;
+  return AS_OK;
+}
+
 extern "C" {
 
 const char* as_status_string(as_status_t s) {
@@ -174,6 +190,11 @@ as_status_t as_hybrid_attn_destroy(as_hybrid_attn_t h) {
   if (h->d_sm_rank) cudaFree(h->d_sm_rank);
   if (h->d_status) cudaFree(h->d_status);
   for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
+  for (cudaEvent_t e : h->ev_run) cudaEventDestroy(e);
+  if (h->side_ready) {
+    cudaEventDestroy(h->ev_fork); cudaEventDestroy(h->ev_join);
+    cudaStreamDestroy(h->s_in); cudaStreamDestroy(h->s_out);
+  }
   delete h;
   return AS_OK;
 }
@@ -206,27 +227,37 @@ as_status_t as_hybrid_attn_forward(as_hybrid_attn_t h, const void* q, const void
                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
   if (!h || !q || !k || !v || !out) return AS_ERR_INVALID_ARG;
   const auto& d = h->desc;
-  const bool lin = h->n_l > 0;
-  if (lin) {
-    if (!w || !w->wq1 || !w->wk1) return AS_ERR_INVALID_ARG;
-    if (w->bq1 || w->bk1 || w->bq2 || w->bk2) return AS_ERR_UNSUPPORTED;
-    if (d.phi_layers == 1 && (w->wq2 || w->wk2)) return AS_ERR_INVALID_ARG;
-    if (d.phi_layers == 2 && (!w->wq2 || !w->wk2)) return AS_ERR_INVALID_ARG;
-    if (((uintptr_t)w->wq1 | (uintptr_t)w->wk1 | (uintptr_t)w->wq2 | (uintptr_t)w->wk2) & 15) return AS_ERR_INVALID_ARG;
-  }
+  const as_status_t ws_ok = check_weights(h, w);
+  if (ws_ok != AS_OK) return ws_ok;
   if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15) return AS_ERR_INVALID_ARG;
   if (aux && ((uintptr_t)aux & 3)) return AS_ERR_INVALID_ARG;
   if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < h->ws.total) return AS_ERR_WORKSPACE;
-  cudaStream_t st = (cudaStream_t)cuda_stream;
-  char* ws = (char*)workspace;
+  return launch_heads(h, q, k, v, w, out, aux, (char*)workspace, (cudaStream_t)cuda_stream, 0, d.B * d.H, d.B, d.H);
+}
 
+}  // extern "C"
+
+// Launches the kernels for `count` consecutive (batch, head) pairs starting at global pair `first`
+// (all of them, or a run of heads inside one batch entry).  q, k, v, out, aux point at the first pair of
+// the run; the run is presented to the kernels as nb x nh pairs (nb * nh == count).  Scratch that only
+// lives inside one forward (compacted K/V, partial sums) is shared by all runs; S, z and the bf16 S keep
+// their place in the full [B*H] arrays, so linear_state sees every pair afterwards.
+static as_status_t launch_heads(as_hybrid_attn_t h, const void* q, const void* k, const void* v,
+                                const as_phi_weights_t* w, void* out, float* aux, char* ws, cudaStream_t st,
+                                int first, int count, int nb, int nh) {
+  const auto& d = h->desc;
+  const bool lin = h->n_l > 0;
+  const int head0 = first % d.H;                 // the run's first head: where its weights start
+  const size_t F = d.phi_dim, dd = d.d;
+  (void)count;
   as_launch_args a{};
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;
-  a.wq = lin ? (const __nv_bfloat16*)w->wq1 : nullptr;
-  a.wk = lin ? (const __nv_bfloat16*)w->wk1 : nullptr;
   const bool two = lin && d.phi_layers == 2;
-  a.wq2 = two ? (const __nv_bfloat16*)w->wq2 : nullptr;
-  a.wk2 = two ? (const __nv_bfloat16*)w->wk2 : nullptr;
+  const size_t w1 = (two ? dd : F) * dd;         // elements of one head's first-layer matrix
+  a.wq = lin ? (const __nv_bfloat16*)w->wq1 + head0 * w1 : nullptr;
+  a.wk = lin ? (const __nv_bfloat16*)w->wk1 + head0 * w1 : nullptr;
+  a.wq2 = two ? (const __nv_bfloat16*)w->wq2 + head0 * F * dd : nullptr;
+  a.wk2 = two ? (const __nv_bfloat16*)w->wk2 + head0 * F * dd : nullptr;
   a.h1q = two ? (__nv_bfloat16*)(ws + h->ws.h1q) : nullptr;
   a.h1k = two ? (__nv_bfloat16*)(ws + h->ws.h1k) : nullptr;
   a.layers = d.phi_layers;
@@ -237,10 +268,10 @@ as_status_t as_hybrid_attn_forward(as_hybrid_attn_t h, const void* q, const void
   a.ks = compact ? a.ks_w : a.k;
   a.vs = compact ? a.vs_w : a.v;
   a.part_s = (float*)(ws + h->ws.part_s); a.part_z = (float*)(ws + h->ws.part_z);
-  a.S = (float*)(ws + h->ws.S); a.z = (float*)(ws + h->ws.z);
-  a.Sb = (__nv_bfloat16*)(ws + h->ws.Sb);
+  a.S = (float*)(ws + h->ws.S) + (size_t)first * F * dd; a.z = (float*)(ws + h->ws.z) + (size_t)first * F;
+  a.Sb = (__nv_bfloat16*)(ws + h->ws.Sb) + (size_t)first * F * dd;
   a.sm_rank = h->d_sm_rank; a.status = h->d_status;
-  a.B = d.B; a.H = d.H; a.N = d.N; a.d = d.d; a.F = d.phi_dim; a.P = d.poly_degree;
+  a.B = nb; a.H = nh; a.N = d.N; a.d = d.d; a.F = d.phi_dim; a.P = d.poly_degree;
   a.n_s = h->n_s; a.n_l = h->n_l; a.n_chunks = h->n_chunks; a.chunk_tiles = h->chunk_tiles;
   a.scale = h->scale; a.stab_mode = d.stab_mode;
 
@@ -265,6 +296,8 @@ as_status_t as_hybrid_attn_forward(as_hybrid_attn_t h, const void* q, const void
   return AS_OK;
 }
 
+extern "C" {
+
 as_status_t as_hybrid_attn_forward_host(as_hybrid_attn_t h, const void* q_host, const void* k_host,
                                         const void* v_host, const as_phi_weights_t* w,
                                         void* out_host, void* workspace, size_t workspace_bytes,
@@ -272,20 +305,59 @@ as_status_t as_hybrid_attn_forward_host(as_hybrid_attn_t h, const void* q_host, 
   if (!h || !q_host || !k_host || !v_host || !out_host) return AS_ERR_INVALID_ARG;
   if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < h->ws.total_host) return AS_ERR_WORKSPACE;
   const auto& d = h->desc;
-  const size_t bytes = (size_t)d.B * d.H * d.N * d.d * 2;
+  const as_status_t ws_ok = check_weights(h, w);
+  if (ws_ok != AS_OK) return ws_ok;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   char* ws = (char*)workspace;
-  if (cudaMemcpyAsync(ws + h->ws.stage_q, q_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(ws + h->ws.stage_k, k_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(ws + h->ws.stage_v, v_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
-    cudaGetLastError(); return AS_ERR_CUDA;
+  // The three copies in, the kernels and the copy out of one run of heads form a pipeline over runs:
+  // copies in on one side stream, kernels on the caller's stream, copies out on another side stream, so
+  // that both directions of the host link and the kernels work at the same time.  A run is a whole
+  // number of heads of one batch entry with at least ~8 MB of q.
+  const size_t head_bytes = (size_t)d.N * d.d * 2;
+  int run = (int)std::min<size_t>((size_t)d.H, std::max<size_t>(1, ((size_t)8 << 20) / head_bytes));
+  const int runs_per_batch = (d.H + run - 1) / run;
+  const int n_runs = d.B * runs_per_batch;
+  if (!h->side_ready) {
+    if (cudaStreamCreateWithFlags(&h->s_in, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&h->s_out, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+      cudaGetLastError(); return AS_ERR_CUDA;
+    }
+    h->side_ready = true;
   }
-  as_status_t s = as_hybrid_attn_forward(h, ws + h->ws.stage_q, ws + h->ws.stage_k, ws + h->ws.stage_v, w,
-                                         ws + h->ws.stage_o, nullptr, workspace, h->ws.total, cuda_stream);
-  if (s != AS_OK) return s;
-  if (cudaMemcpyAsync(out_host, ws + h->ws.stage_o, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
-    cudaGetLastError(); return AS_ERR_CUDA;
+  while ((int)h->ev_run.size() < 2 * n_runs) {
+    cudaEvent_t e;
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
+    h->ev_run.push_back(e);
   }
+  bool ok = cudaEventRecord(h->ev_fork, st) == cudaSuccess &&
+            cudaStreamWaitEvent(h->s_in, h->ev_fork, 0) == cudaSuccess &&
+            cudaStreamWaitEvent(h->s_out, h->ev_fork, 0) == cudaSuccess;
+  as_status_t status = AS_OK;
+  for (int r = 0; ok && r < n_runs; ++r) {
+    const int b = r / runs_per_batch, h0 = (r % runs_per_batch) * run;
+    const int nh = std::min(run, d.H - h0);
+    const int first = b * d.H + h0;
+    const size_t off = (size_t)first * head_bytes, bytes = (size_t)nh * head_bytes;
+    cudaEvent_t ev_in = h->ev_run[2 * r], ev_done = h->ev_run[2 * r + 1];
+    ok = cudaMemcpyAsync(ws + h->ws.stage_q + off, (const char*)q_host + off, bytes, cudaMemcpyHostToDevice, h->s_in) == cudaSuccess &&
+         cudaMemcpyAsync(ws + h->ws.stage_k + off, (const char*)k_host + off, bytes, cudaMemcpyHostToDevice, h->s_in) == cudaSuccess &&
+         cudaMemcpyAsync(ws + h->ws.stage_v + off, (const char*)v_host + off, bytes, cudaMemcpyHostToDevice, h->s_in) == cudaSuccess &&
+         cudaEventRecord(ev_in, h->s_in) == cudaSuccess && cudaStreamWaitEvent(st, ev_in, 0) == cudaSuccess;
+    if (!ok) break;
+    status = launch_heads(h, ws + h->ws.stage_q + off, ws + h->ws.stage_k + off, ws + h->ws.stage_v + off, w,
+                          ws + h->ws.stage_o + off, nullptr, ws, st, first, nh, 1, nh);
+    if (status != AS_OK) break;
+    ok = cudaEventRecord(ev_done, st) == cudaSuccess && cudaStreamWaitEvent(h->s_out, ev_done, 0) == cudaSuccess &&
+         cudaMemcpyAsync((char*)out_host + off, ws + h->ws.stage_o + off, bytes, cudaMemcpyDeviceToHost, h->s_out) == cudaSuccess;
+  }
+  // join: the caller's stream completes only after the last copy out (and, after an error, after
+  // whatever the side streams were already given)
+  const bool joined = cudaEventRecord(h->ev_join, h->s_out) == cudaSuccess && cudaStreamWaitEvent(st, h->ev_join, 0) == cudaSuccess &&
+                      cudaEventRecord(h->ev_fork, h->s_in) == cudaSuccess && cudaStreamWaitEvent(st, h->ev_fork, 0) == cudaSuccess;
+  if (status != AS_OK) return status;
+  if (!ok || !joined) { cudaGetLastError(); return AS_ERR_CUDA; }
   return AS_OK;
 }
 

@@ -60,6 +60,11 @@ struct as_hybrid_attn_s {
   std::vector<cudaEvent_t> ev;          // 2 * AS_MAX_PROFILE events, created on first enable
   std::vector<int> ev_class;
   int ev_used = 0;
+  // forward_host: side streams for the copies in and out, created on its first call
+  bool side_ready = false;
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  std::vector<cudaEvent_t> ev_run;      // per run of heads: inputs landed, kernels done
 };
 
 // Kernel launchers.  Each returns the launch's cudaError_t.

@@ -720,9 +720,11 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         if (lane == 0) sMask[b * 4 + warp] = bits;
         lin_next = is_linear(t + 1);
       }
+      // every feature thread reaches this barrier in every iteration, also after a failed wait: a warp
+      // that left the loop early would leave the others waiting here for good
       named_barrier_sync(1, 128);
-      ok = mbar_wait_warp(bar(B_D1 + b), (t >> 1) & 1, wc);
-      if (!ok) break;
+      if (ok) ok = mbar_wait_warp(bar(B_D1 + b), (t >> 1) & 1, wc);
+      if (!ok) continue;
       tc_fence_after();
 #pragma unroll
       for (int c = 0; c < 4; ++c) {

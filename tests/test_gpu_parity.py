@@ -397,3 +397,27 @@ def test_two_layer_needs_its_second_weights_and_the_tensor_path():
     with pytest.raises(AsError) as e:
         op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"])
     assert e.value.status == binding.AS_ERR_INVALID_ARG
+
+
+def test_host_entry_point_pipelined_over_runs_of_heads():
+    """Large enough that the host entry point works in several runs of heads (copies in, kernels and
+    copies out overlapped): same bits as the device entry point, and the linear state of every head is
+    in place afterwards."""
+    import torch
+    from paper_2509_24899_b200 import HybridAttention
+    wl = W.Workload("host_runs", B=2, H=3, d=128, F=128, grid=(4, 64, 64), block=(2, 4, 4), rate=8, seed=21)
+    data = W.generate(wl, wq_gain=0.02)
+    dev = {k: to_cuda_bf16(v) for k, v in data.items()}
+    op = HybridAttention.from_workload(wl, kernel_path=_path(FULL_PATH))
+    ref = op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"]).clone()
+    S_ref, z_ref = (t.clone() for t in op.linear_state())
+    host = {k: torch.from_numpy(data[k].view(np.int16)).pin_memory() for k in ("q", "k", "v")}
+    out_host = torch.zeros_like(host["q"]).pin_memory()
+    for _ in range(2):                                   # the second call reuses the side streams and events
+        out_host.zero_()
+        op.forward_host(host["q"], host["k"], host["v"], dev["wq"], dev["wk"], out_host)
+        torch.cuda.synchronize()
+        assert op.last_status() == 0
+        assert torch.equal(out_host, ref.view(torch.int16).cpu())
+        S, z = op.linear_state()
+        assert torch.equal(S, S_ref) and torch.equal(z, z_ref)
