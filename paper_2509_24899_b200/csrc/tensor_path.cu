@@ -134,6 +134,20 @@ struct QRing {
   AS_DEV bool wait(int b, int phase) const { return mbar_wait_warp(bar(b), phase & 1, c.wc); }
   AS_DEV bool full_wait(int item) const { return wait(B_FULL + item % KV_STAGES, item / KV_STAGES); }
   AS_DEV void release(int item) const { tc_commit(bar(B_EMPTY + item % KV_STAGES)); }
+  // single-thread forms for the issuing thread (no warp vote): a wait that is already satisfied still
+  // costs a round trip to shared memory, so barriers needed together are probed together
+  AS_DEV bool wait1(int b, int phase) const { return mbar_wait(bar(b), phase & 1, c.wc); }
+  AS_DEV bool probe(int b, int phase) const { return mbar_try_wait(bar(b), phase & 1); }
+  AS_DEV int full_bar(int item) const { return B_FULL + item % KV_STAGES; }
+  AS_DEV bool wait3(int b0, int ph0, bool use1, int b1, int ph1, bool use2, int b2, int ph2) const {
+    const bool r0 = probe(b0, ph0);
+    const bool r1 = use1 ? probe(b1, ph1) : true;
+    const bool r2 = use2 ? probe(b2, ph2) : true;
+    if (r0 && r1 && r2) return true;
+    if (!r1 && !wait1(b1, ph1)) return false;
+    if (!r2 && !wait1(b2, ph2)) return false;
+    return r0 || wait1(b0, ph0);
+  }
 };
 
 // ---------------------------------------------------------------- TMA producer, one unit
@@ -182,6 +196,10 @@ __device__ __noinline__ bool q_produce_unit(const QParams& p, const QCtx& c, con
 }
 
 // ---------------------------------------------------------------- MMA issuer, one unit
+// Runs in ONE thread (lane 0 of the issuing warp; the other lanes wait at the end of the role): this
+// thread is the busiest resource of the CTA - every clock it spends outside the MMA instructions is a
+// clock the tensor pipe idles - so it takes no warp votes or warp barriers, probes the barriers it needs
+// together, and has its operands ready before it looks at a barrier.
 template <int D>
 __device__ __noinline__ bool q_mma_unit(const QParams& p, const QCtx& c, int u) {
   using R = QRing<D>;
@@ -191,31 +209,27 @@ __device__ __noinline__ bool q_mma_unit(const QParams& p, const QCtx& c, int u) 
   constexpr uint32_t ID_PHI = make_idesc(128, F, 0, 0);       // Phi = Q W_q^T  (N = F)
   const int nkv = p.nkv, lin = p.lin, layers = p.layers;
   const R q(nkv, lin, layers, c);
-  const int lane = threadIdx.x & 31;
   const int base = u * q.n_items, pb = u * q.n_sp;            // first ring item / first S,P phase of the unit
-  if (!q.wait(R::B_Q0, u)) return false;
-  if (nkv == 0 && !q.wait(R::B_Q0 + 1, u)) return false;
-  if (nkv > 0) {
-    if (!q.full_wait(base)) return false;
+  if (nkv == 0) {
+    if (!q.wait1(R::B_Q0, u) || !q.wait1(R::B_Q0 + 1, u)) return false;
+  } else {
+    if (!q.wait3(R::B_Q0, u, true, q.full_bar(base), base / KV_STAGES, false, 0, 0)) return false;
     for (int g = 0; g < 2; ++g) {
-      if (g == 1 && !q.wait(R::B_Q0 + 1, u)) return false;
+      if (g == 1 && !q.wait1(R::B_Q0 + 1, u)) return false;
       tc_fence_after();
-      if (lane == 0) {
-        issue_kmajor<D>(q.tS(g), kmajor_desc(q.sQ(g)), kmajor_desc(q.sKV(base)), ID_QK, false);
-        tc_commit(q.bar(R::B_S + g));
-        if (g == 1) q.release(base);
-      }
-      __syncwarp();
+      issue_kmajor<D>(q.tS(g), kmajor_desc(q.sQ(g)), kmajor_desc(q.sKV(base)), ID_QK, false);
+      tc_commit(q.bar(R::B_S + g));
+      if (g == 1) q.release(base);
     }
     for (int j = 0; j < nkv; ++j) {
       // this tile's V; the next tile's K, or after the last tile the feature weights: Phi = X W^T is
       // issued right behind the group's last P V, in the place the next tile's Q K^T would have
       const bool last = (j + 1 == nkv);
+      const bool more = !last || lin;                         // a score-like product follows the P V
       const int iv = base + 2 * j + 1, ik = last ? base + q.it_w : base + 2 * j + 2;
       const uint32_t id_next = last ? ID_PHI : ID_QK;
 #pragma unroll
       for (int g = 0; g < 2; ++g) {
-        // operands of the whole block are prepared before the wait, so that the issue itself is short
         uint64_t dv[8], dq[8], dk[8];
         uint32_t ap[8];
         {
@@ -230,68 +244,56 @@ __device__ __noinline__ bool q_mma_unit(const QParams& p, const QCtx& c, int u) 
             ap[kk] = q.tS(g) + kk * 8;
           }
         }
-        if (!q.wait(R::B_P + g, pb + j)) return false;
-        if (g == 0 && !q.full_wait(iv)) return false;
-        if (g == 0 && (!last || lin) && !q.full_wait(ik)) return false;
-        if (last && layers == 2 && !q.full_wait(base + q.it_h + g)) return false;
+        // P of this group and tile, and (first group only) the two ring tiles the block reads
+        if (!q.wait3(R::B_P + g, pb + j, g == 0, q.full_bar(iv), iv / KV_STAGES, g == 0 && more, q.full_bar(ik), ik / KV_STAGES))
+          return false;
+        if (last && layers == 2 && !q.wait1(q.full_bar(base + q.it_h + g), (base + q.it_h + g) / KV_STAGES)) return false;
         tc_fence_after();
-        if (lane == 0) {
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) mma_ts(q.tO(g), ap[kk], dv[kk], ID_PV, (j > 0 || kk > 0) ? 1u : 0u);
-          if (!last || lin) {
+        for (int kk = 0; kk < 8; ++kk) mma_ts(q.tO(g), ap[kk], dv[kk], ID_PV, (j > 0 || kk > 0) ? 1u : 0u);
+        if (more) {
 #pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), dq[kk], dk[kk], id_next, kk > 0 ? 1u : 0u);
-            tc_commit(q.bar(R::B_S + g));
-          } else {
-            tc_commit(q.bar(R::B_O + g));
-          }
-          if (last) {
-            tc_commit(q.bar(R::B_QF + g));           // nothing of this unit reads the group's Q tile any more
-            if (layers == 2) q.release(base + q.it_h + g);
-          }
+          for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), dq[kk], dk[kk], id_next, kk > 0 ? 1u : 0u);
+          tc_commit(q.bar(R::B_S + g));
+        } else {
+          tc_commit(q.bar(R::B_O + g));
         }
-        __syncwarp();
+        if (last) {
+          tc_commit(q.bar(R::B_QF + g));             // nothing of this unit reads the group's Q tile any more
+          if (layers == 2) q.release(base + q.it_h + g);
+        }
       }
-      if (lane == 0) {
-        q.release(iv);
-        if (!last || lin) q.release(ik);
-      }
-      __syncwarp();
+      q.release(iv);
+      if (more) q.release(ik);
     }
   }
   if (lin && nkv == 0) {
     // no softmax tokens at all: the feature product opens the unit
-    if (!q.full_wait(base + q.it_w)) return false;
+    if (!q.wait1(q.full_bar(base + q.it_w), (base + q.it_w) / KV_STAGES)) return false;
     for (int g = 0; g < 2; ++g) {
       // Phi = X W^T with X = Q (one layer) or the first-layer activations (two layers)
-      if (layers == 2 && !q.full_wait(base + q.it_h + g)) return false;
+      if (layers == 2 && !q.wait1(q.full_bar(base + q.it_h + g), (base + q.it_h + g) / KV_STAGES)) return false;
       tc_fence_after();
-      if (lane == 0) {
-        issue_kmajor<D>(q.tS(g), kmajor_desc(layers == 2 ? q.sKV(base + q.it_h + g) : q.sQ(g)),
-                        kmajor_desc(q.sKV(base + q.it_w)), ID_PHI, false);
-        tc_commit(q.bar(R::B_S + g));
-        tc_commit(q.bar(R::B_QF + g));               // nothing of this unit reads the group's Q tile any more
-        if (layers == 2) q.release(base + q.it_h + g);
-        if (g == 1) q.release(base + q.it_w);
-      }
-      __syncwarp();
+      issue_kmajor<D>(q.tS(g), kmajor_desc(layers == 2 ? q.sKV(base + q.it_h + g) : q.sQ(g)),
+                      kmajor_desc(q.sKV(base + q.it_w)), ID_PHI, false);
+      tc_commit(q.bar(R::B_S + g));
+      tc_commit(q.bar(R::B_QF + g));                 // nothing of this unit reads the group's Q tile any more
+      if (layers == 2) q.release(base + q.it_h + g);
+      if (g == 1) q.release(base + q.it_w);
     }
   }
   if (lin) {
-    if (!q.full_wait(base + q.it_st)) return false;
+    const int is = base + q.it_st;
     for (int g = 0; g < 2; ++g) {
-      if (!q.wait(R::B_P + g, pb + nkv)) return false;
+      if (!q.wait3(R::B_P + g, pb + nkv, g == 0, q.full_bar(is), is / KV_STAGES, false, 0, 0)) return false;
       tc_fence_after();
-      if (lane == 0) {
-        // phi_q sits where P sits (bf16 over the score columns), S plays the part of a V tile
-        const uint64_t s0 = mnmajor_desc(q.sKV(base + q.it_st));
+      // phi_q sits where P sits (bf16 over the score columns), S plays the part of a V tile
+      const uint64_t s0 = mnmajor_desc(q.sKV(is));
 #pragma unroll
-        for (int kk = 0; kk < F / 16; ++kk)
-          mma_ts(q.tO(g), q.tS(g) + kk * 8, s0 + (uint64_t)((kk * 2048) >> 4), ID_PV, (nkv > 0 || kk > 0) ? 1u : 0u);
-        tc_commit(q.bar(R::B_O + g));
-        if (g == 1) q.release(base + q.it_st);
-      }
-      __syncwarp();
+      for (int kk = 0; kk < F / 16; ++kk)
+        mma_ts(q.tO(g), q.tS(g) + kk * 8, s0 + (uint64_t)((kk * 2048) >> 4), ID_PV, (nkv > 0 || kk > 0) ? 1u : 0u);
+      tc_commit(q.bar(R::B_O + g));
+      if (g == 1) q.release(is);
     }
   }
   return true;
@@ -506,8 +508,11 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     for (int u = 0; u < n_mine; ++u)
       if (!q_produce_unit<D>(p, c, &tmQ, &tmK, &tmV, &tmW, &tmSt, &tmH, u)) break;
   } else if (warp == 9) {
-    for (int u = 0; u < n_mine; ++u)
-      if (!q_mma_unit<D>(p, c, u)) break;
+    if ((threadIdx.x & 31) == 0) {
+      for (int u = 0; u < n_mine; ++u)
+        if (!q_mma_unit<D>(p, c, u)) break;
+    }
+    __syncwarp();
   } else {
     for (int u = 0; u < n_mine; ++u)
       if (!q_softmax_unit<D>(p, c, &tmO, smem, u)) break;
