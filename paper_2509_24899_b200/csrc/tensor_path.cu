@@ -8,11 +8,14 @@
 //     softmax-token rows of the K / V tiles are copied from shared memory to the compact K_S / V_S.
 //   Q pass  (steps: softmax branch, phi_q projection, linear apply, merge)
 //     persistent, one CTA per SM; per unit of 2 x 128 query rows a flash-style loop over 128-key tiles
-//     of K_S / V_S:        S = Q K_S^T -> TMEM, running max / sum per row (one thread per row),
-//                          P = exp2(.) as bf16 back into TMEM, O += P V_S (TMEM x smem)
-//     tail:                Phi = Q W_q^T -> TMEM (issued right behind the last P V), phi_q scaled per row
-//                          as bf16 where P sat, O += phi_q S (TMEM x smem, S in bf16 read like a V tile),
-//                          den = l + phi_q.z, y = O / den -> bf16 -> per-warp staging -> TMA store.
+//     of K_S / V_S:        S = Q K_S^T -> TMEM; the softmax threads (one per row) read their row and
+//                          release the score columns at once, so the next tile's Q K_S^T runs under the
+//                          exponentials; running max / sum per row; P = exp2(.) as bf16 -> shared memory,
+//                          O += P V_S (smem x smem -> TMEM).  Two issuing threads: one for what writes
+//                          the score columns, one for what accumulates into O.
+//     tail:                Phi = Q W_q^T -> TMEM (in the place of a next tile's scores), phi_q scaled per
+//                          row as bf16 where P sat, O += phi_q S (S in bf16 read like a V tile),
+//                          den = l + phi_q.z, y = O / den -> bf16 -> staged in the P tile -> TMA store.
 // All tiles are staged by TMA with the 128-byte swizzle; every mbarrier wait is bounded.
 #include <cuda.h>
 
@@ -41,18 +44,18 @@ struct QParams {
   uint32_t* status;
 };
 
-constexpr int Q_THREADS = 320;           // warps 0-3 / 4-7: softmax groups 0 / 1; warp 8: TMA; warp 9: MMA
-constexpr int KV_STAGES = 4;
+constexpr int Q_THREADS = 352;           // warps 0-3 / 4-7: softmax groups 0 / 1; warp 8: TMA; warps 9, 10: MMA issuers
+constexpr int KV_STAGES = 3;
 constexpr float RESCALE_THRESHOLD = 8.f; // log2 units: rescale O only when the row max grew by > 2^8
 
 template <int D>
 struct QLayout {
   static constexpr int TILE = 128 * D * 2;                 // bytes of a [128 x D] bf16 tile
+  static constexpr int PTILE = 128 * 128 * 2;              // bytes of a [128 rows x 128 keys] bf16 P tile
   static constexpr int Q_OFF = 0;
-  static constexpr int KV_OFF = 2 * TILE;
-  static constexpr int OUT_OFF = KV_OFF + KV_STAGES * TILE;  // per softmax warp: 32 rows x 64 columns of bf16 output
-  static constexpr int OUT_WARP = 32 * 128;
-  static constexpr int BAR_OFF = OUT_OFF + 8 * OUT_WARP;
+  static constexpr int P_OFF = 2 * TILE;                   // per group: P, then phi_q, then the output rows
+  static constexpr int KV_OFF = P_OFF + 2 * PTILE;
+  static constexpr int BAR_OFF = KV_OFF + KV_STAGES * TILE;
   static constexpr int TOTAL = BAR_OFF + 256 + 1024;       // + slack for the 1024-byte alignment
 };
 
@@ -67,21 +70,23 @@ AS_DEV void load_tile(uint32_t dst, const CUtensorMap* m, uint32_t bar, int y0, 
 // offset (in 16-byte units) to the address field, which keeps the issuing thread's instruction count low.
 AS_DEV uint64_t kmajor_desc(uint32_t smem) { return make_sdesc(smem, 16, 1024); }        // [rows x 64] boxes, K-major
 AS_DEV uint64_t mnmajor_desc(uint32_t smem) { return make_sdesc(smem, BOX_BYTES, 1024); } // k-rows x [64-column boxes], MN-major
+// offset of k-step kk (16 elements) inside a K-major tile of 64-column boxes
+AS_DEV constexpr uint64_t kstep_kmajor(int kk) { return (uint64_t)(((kk / 4) * BOX_BYTES + (kk % 4) * 32) >> 4); }
+// offset of k-step kk (16 rows) inside an MN-major tile
+AS_DEV constexpr uint64_t kstep_mnmajor(int kk) { return (uint64_t)((kk * 2048) >> 4); }
 
 // D[tmem] (+)= A[smem, K-major, 128 x KD] * B[smem, K-major, NB x KD]^T
 template <int KD>
 AS_DEV void issue_kmajor(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool acc) {
 #pragma unroll
-  for (int kk = 0; kk < KD / 16; ++kk) {
-    const uint64_t off = (uint64_t)(((kk / 4) * BOX_BYTES + (kk % 4) * 32) >> 4);
-    mma_ss(d_tmem, a_desc + off, b_desc + off, idesc, (acc || kk > 0) ? 1u : 0u);
-  }
+  for (int kk = 0; kk < KD / 16; ++kk)
+    mma_ss(d_tmem, a_desc + kstep_kmajor(kk), b_desc + kstep_kmajor(kk), idesc, (acc || kk > 0) ? 1u : 0u);
 }
 // D[tmem] (+)= A[tmem, 128 lanes x 128 k as packed bf16] * B[smem, MN-major: 128 k-rows x NB cols]
 AS_DEV void issue_tmemA_mnB(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool acc) {
 #pragma unroll
   for (int kk = 0; kk < 8; ++kk)
-    mma_ts(d_tmem, a_tmem + kk * 8, b_desc + (uint64_t)((kk * 2048) >> 4), idesc, (acc || kk > 0) ? 1u : 0u);
+    mma_ts(d_tmem, a_tmem + kk * 8, b_desc + kstep_mnmajor(kk), idesc, (acc || kk > 0) ? 1u : 0u);
 }
 
 // Writes 32 consecutive columns [c0, c0+32) of row `row` of a swizzled [128 x D] bf16 tile.
@@ -97,9 +102,13 @@ AS_DEV void store_row_chunk(uint8_t* tile, uint32_t row, uint32_t c0, const uint
 
 // Persistent: one CTA per SM walks over 256-row units (unit w = blockIdx.x + u * gridDim.x; the units of
 // one (batch, head) are consecutive, so the CTAs that run at the same time share K_S / V_S in L2).
-// Barrier phases and the K/V ring run on across units: the producer prefetches the next unit's first
-// key tiles and its Q tiles (as soon as the linear apply has released the Q buffer) while the softmax
-// warps still normalise and store the previous unit.
+// Barrier phases and the K/V ring run on across units.
+//
+// Scores and probabilities live in different memories: S = Q K^T lands in TMEM, the softmax threads read
+// their rows into registers and release the S columns at once, so the next tile's Q K^T is computed while
+// the exponentials run; P goes to shared memory as bf16 and is the A operand of O += P V.  A group's
+// softmax therefore never waits for the tensor pipe in the steady state, and the pipe sees, per key tile
+// and group, one Q K^T block as soon as S is free and one P V block as soon as P is there.
 //
 // The work of one unit is a function per role, kept out of line: each role then gets a register
 // allocation of its own (the softmax rows need nearly the whole budget, and the issuing thread must
@@ -113,39 +122,49 @@ struct QCtx {
 template <int D>
 struct QRing {
   using L = QLayout<D>;
-  // barrier indices
-  static constexpr int B_Q0 = 0, B_FULL = 2, B_EMPTY = 2 + KV_STAGES, B_S = 2 + 2 * KV_STAGES, B_P = B_S + 2,
-                       B_O = B_P + 2, B_QF = B_O + 2, B_COUNT = B_QF + 2;
+  // barrier indices; per group: S (scores or Phi landed), SF (score columns read out), P (P or phi_q in
+  // shared memory), PF (the product that reads the P buffer has completed), O (output accumulator final),
+  // QF (nothing of the unit reads the Q tile any more)
+  static constexpr int B_Q0 = 0, B_FULL = 2, B_EMPTY = B_FULL + KV_STAGES, B_S = B_EMPTY + KV_STAGES, B_SF = B_S + 2,
+                       B_P = B_SF + 2, B_PF = B_P + 2, B_O = B_PF + 2, B_QF = B_O + 2, B_COUNT = B_QF + 2;
   const QCtx c;              // by value: nothing here is re-read from memory after a barrier or an MMA
-  int it_w, it_h, it_st, n_items, n_sp;
-  // items of one unit: K and V tiles alternating, then for the linear tail the last-layer weights,
-  // (with a two-layer feature map) the two groups' first-layer activations, and S in bf16
-  AS_DEV QRing(int nkv, int lin, int layers, const QCtx& c_) : c(c_) {
-    it_w = 2 * nkv; it_h = 2 * nkv + 1; it_st = 2 * nkv + (layers == 2 ? 3 : 1);
-    n_items = lin ? it_st + 1 : 2 * nkv;
-    n_sp = nkv + lin;                    // completions of the S and of the P barrier per unit and group
+  int nkv, lin, two;
+  int it_h, it_w, it_vlast, it_st, n_items, n_sp;
+  // Ring items of one unit, in the order they are consumed: K_0; then K_{j+1}, V_j for j = 0 .. nkv-2;
+  // then for the linear tail (two-layer map: the two groups' first-layer activations,) the last-layer
+  // weights; V_{nkv-1}; S in bf16.
+  AS_DEV QRing(int nkv_, int lin_, int layers, const QCtx& c_) : c(c_), nkv(nkv_), lin(lin_), two(lin_ && layers == 2) {
+    int next = nkv > 0 ? 2 * nkv - 1 : 0;
+    it_h = next; if (two) next += 2;
+    it_w = next; if (lin) next += 1;
+    it_vlast = next; if (nkv > 0) next += 1;
+    it_st = next; if (lin) next += 1;
+    n_items = next;
+    n_sp = nkv + lin;                    // per unit and group: S completions = P hand-overs = P-buffer releases
   }
+  AS_DEV int item_k(int j) const { return j == 0 ? 0 : 2 * j - 1; }
+  AS_DEV int item_v(int j) const { return j + 1 < nkv ? 2 * j + 2 : it_vlast; }
   AS_DEV uint32_t bar(int i) const { return c.sbase + L::BAR_OFF + 8 * i; }
   AS_DEV uint32_t sQ(int g) const { return c.sbase + L::Q_OFF + g * L::TILE; }
+  AS_DEV uint32_t sP(int g) const { return c.sbase + L::P_OFF + g * L::PTILE; }
   // The K/V ring is indexed by a running item number that does not restart with a unit.
   AS_DEV uint32_t sKV(int item) const { return c.sbase + L::KV_OFF + (item % KV_STAGES) * L::TILE; }
   AS_DEV uint32_t tS(int g) const { return c.tmem + 128u * g; }
   AS_DEV uint32_t tO(int g) const { return c.tmem + 256u + 128u * g; }
   AS_DEV bool wait(int b, int phase) const { return mbar_wait_warp(bar(b), phase & 1, c.wc); }
-  AS_DEV bool full_wait(int item) const { return wait(B_FULL + item % KV_STAGES, item / KV_STAGES); }
   AS_DEV void release(int item) const { tc_commit(bar(B_EMPTY + item % KV_STAGES)); }
   // single-thread forms for the issuing thread (no warp vote): a wait that is already satisfied still
   // costs a round trip to shared memory, so barriers needed together are probed together
   AS_DEV bool wait1(int b, int phase) const { return mbar_wait(bar(b), phase & 1, c.wc); }
   AS_DEV bool probe(int b, int phase) const { return mbar_try_wait(bar(b), phase & 1); }
-  AS_DEV int full_bar(int item) const { return B_FULL + item % KV_STAGES; }
-  AS_DEV bool wait3(int b0, int ph0, bool use1, int b1, int ph1, bool use2, int b2, int ph2) const {
+  AS_DEV bool wait_full(int item) const { return wait1(B_FULL + item % KV_STAGES, item / KV_STAGES); }
+  // barrier b0 and, when use1, the ring item's full barrier
+  AS_DEV bool wait2(int b0, int ph0, bool use1, int item) const {
+    const int b1 = B_FULL + item % KV_STAGES, ph1 = item / KV_STAGES;
     const bool r0 = probe(b0, ph0);
     const bool r1 = use1 ? probe(b1, ph1) : true;
-    const bool r2 = use2 ? probe(b2, ph2) : true;
-    if (r0 && r1 && r2) return true;
+    if (r0 && r1) return true;
     if (!r1 && !wait1(b1, ph1)) return false;
-    if (!r2 && !wait1(b2, ph2)) return false;
     return r0 || wait1(b0, ph0);
   }
 };
@@ -163,7 +182,8 @@ __device__ __noinline__ bool q_produce_unit(const QParams& p, const QCtx& c, con
   const int w = (int)blockIdx.x + u * (int)gridDim.x;
   const int bh = w / p.nx, h = bh % p.H, row0 = (w % p.nx) * 256;
   const int base = u * q.n_items;
-  const int q_at = nkv > 0 ? 2 : 0;         // the Q tiles are requested after the unit's first K and V tile
+  const int n_stream = nkv > 0 ? 2 * nkv - 1 : 0;     // K_0, then K_{j+1}, V_j alternating
+  const int q_at = nkv > 0 ? 1 : 0;                   // the Q tiles are requested right after the unit's first K tile
   for (int it = 0; it < q.n_items; ++it) {
     if (it == q_at) {
       for (int g = 0; g < 2; ++g) {
@@ -180,14 +200,18 @@ __device__ __noinline__ bool q_produce_unit(const QParams& p, const QCtx& c, con
     if (!q.wait(R::B_EMPTY + st, gi / KV_STAGES + 1)) return false;
     if (lane == 0) {
       mbar_expect_tx(q.bar(R::B_FULL + st), L::TILE);
-      if (it < 2 * nkv) {
-        load_tile<D>(q.sKV(gi), (it & 1) ? tmV : tmK, q.bar(R::B_FULL + st), (it >> 1) * 128, bh);
-      } else if (it == q.it_w) {
-        load_tile<D>(q.sKV(gi), tmW, q.bar(R::B_FULL + st), 0, h);           // last-layer W_q[h]: [F rows][D]
-      } else if (it < q.it_st) {
-        load_tile<D>(q.sKV(gi), tmH, q.bar(R::B_FULL + st), row0 + (it - q.it_h) * 128, bh);   // relu(q W_1^T) of group it - it_h
+      const uint32_t fb = q.bar(R::B_FULL + st);
+      if (it < n_stream) {
+        if (it == 0 || (it & 1)) load_tile<D>(q.sKV(gi), tmK, fb, ((it + 1) >> 1) * 128, bh);   // K_0 at 0, K_j at 2j-1
+        else load_tile<D>(q.sKV(gi), tmV, fb, ((it >> 1) - 1) * 128, bh);                        // V_j at 2j+2
+      } else if (q.two && it < q.it_w) {
+        load_tile<D>(q.sKV(gi), tmH, fb, row0 + (it - q.it_h) * 128, bh);    // relu(q W_1^T) of group it - it_h
+      } else if (q.lin && it == q.it_w) {
+        load_tile<D>(q.sKV(gi), tmW, fb, 0, h);                              // last-layer W_q[h]: [F rows][D]
+      } else if (nkv > 0 && it == q.it_vlast) {
+        load_tile<D>(q.sKV(gi), tmV, fb, (nkv - 1) * 128, bh);
       } else {
-        load_tile<D>(q.sKV(gi), tmSt, q.bar(R::B_FULL + st), 0, bh);         // S[bh] in bf16: [F rows][D]
+        load_tile<D>(q.sKV(gi), tmSt, fb, 0, bh);                            // S[bh] in bf16: [F rows][D]
       }
     }
     __syncwarp();
@@ -195,103 +219,140 @@ __device__ __noinline__ bool q_produce_unit(const QParams& p, const QCtx& c, con
   return true;
 }
 
-// ---------------------------------------------------------------- MMA issuer, one unit
-// Runs in ONE thread (lane 0 of the issuing warp; the other lanes wait at the end of the role): this
-// thread is the busiest resource of the CTA - every clock it spends outside the MMA instructions is a
-// clock the tensor pipe idles - so it takes no warp votes or warp barriers, probes the barriers it needs
-// together, and has its operands ready before it looks at a barrier.
+// ---------------------------------------------------------------- MMA issuers, one unit
+// Two issuing threads (lane 0 of warps 9 and 10; the other lanes wait at the end of the role): one issues
+// what writes the score columns (Q K^T per tile, Phi at the end) as soon as the softmax threads have read
+// them out, the other what accumulates into O (P V per tile, phi_q S at the end) as soon as P is in
+// shared memory.  The two streams touch different TMEM columns and release different ring items, so they
+// need no ordering between them; each thread's commits cover its own MMAs.  An issuing thread is the
+// busiest resource of the CTA - every clock it spends outside the MMA instructions is a clock the tensor
+// pipe may idle - so it takes no warp votes or warp barriers, probes the barriers it needs together, and
+// has its operands ready before it looks at a barrier.
 template <int D>
-__device__ __noinline__ bool q_mma_unit(const QParams& p, const QCtx& c, int u) {
+__device__ __noinline__ bool q_score_unit(const QParams& p, const QCtx& c, int u) {
   using R = QRing<D>;
   constexpr int F = D;
   constexpr uint32_t ID_QK = make_idesc(128, 128, 0, 0);      // S = Q K^T      (N = 128 keys)
-  constexpr uint32_t ID_PV = make_idesc(128, D, 0, 1);        // O += P V and O += phi_q S  (V, S are MN-major)
   constexpr uint32_t ID_PHI = make_idesc(128, F, 0, 0);       // Phi = Q W_q^T  (N = F)
-  const int nkv = p.nkv, lin = p.lin, layers = p.layers;
-  const R q(nkv, lin, layers, c);
-  const int base = u * q.n_items, pb = u * q.n_sp;            // first ring item / first S,P phase of the unit
-  if (nkv == 0) {
-    if (!q.wait1(R::B_Q0, u) || !q.wait1(R::B_Q0 + 1, u)) return false;
-  } else {
-    if (!q.wait3(R::B_Q0, u, true, q.full_bar(base), base / KV_STAGES, false, 0, 0)) return false;
-    for (int g = 0; g < 2; ++g) {
-      if (g == 1 && !q.wait1(R::B_Q0 + 1, u)) return false;
+  const int nkv = p.nkv, lin = p.lin;
+  const R q(nkv, lin, p.layers, c);
+  const int base = u * q.n_items, pb = u * q.n_sp;            // first ring item / first barrier phase of the unit
+  uint64_t dq[2][8];                                          // the Q tiles do not move within a unit
+#pragma unroll
+  for (int g = 0; g < 2; ++g) {
+    const uint64_t q0 = kmajor_desc(q.sQ(g));
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) dq[g][kk] = q0 + kstep_kmajor(kk);
+  }
+  // Phi = X W^T with X = Q (one layer) or the first-layer activations (two layers), N = F
+  auto issue_phi = [&](int g) {
+    const uint64_t w0 = kmajor_desc(q.sKV(base + q.it_w));
+    if (q.two) {
+      const uint64_t x0 = kmajor_desc(q.sKV(base + q.it_h + g));
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), x0 + kstep_kmajor(kk), w0 + kstep_kmajor(kk), ID_PHI, kk > 0 ? 1u : 0u);
+    } else {
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), dq[g][kk], w0 + kstep_kmajor(kk), ID_PHI, kk > 0 ? 1u : 0u);
+    }
+    tc_commit(q.bar(R::B_S + g));
+    tc_commit(q.bar(R::B_QF + g));                   // nothing of this unit reads the group's Q tile any more
+    if (q.two) q.release(base + q.it_h + g);
+    if (g == 1) q.release(base + q.it_w);
+  };
+  // The first product of a unit overwrites score columns the previous unit's threads read last: wait for
+  // that read (the last S-free phase of the previous unit) together with the Q tile.
+  for (int g = 0; g < 2; ++g) {
+    if (u > 0 && !q.wait1(R::B_SF + g, pb - 1)) return false;
+    if (nkv == 0) {
+      if (!q.wait1(R::B_Q0 + g, u)) return false;
+      if (lin) {
+        // no softmax tokens at all: the feature product opens the unit
+        if (!q.wait_full(base + q.it_w)) return false;
+        if (q.two && !q.wait_full(base + q.it_h + g)) return false;
+        tc_fence_after();
+        issue_phi(g);
+      }
+    } else {
+      if (!q.wait2(R::B_Q0 + g, u, g == 0, base)) return false;
       tc_fence_after();
-      issue_kmajor<D>(q.tS(g), kmajor_desc(q.sQ(g)), kmajor_desc(q.sKV(base)), ID_QK, false);
+      const uint64_t k0 = kmajor_desc(q.sKV(base));
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), dq[g][kk], k0 + kstep_kmajor(kk), ID_QK, kk > 0 ? 1u : 0u);
       tc_commit(q.bar(R::B_S + g));
       if (g == 1) q.release(base);
-    }
-    for (int j = 0; j < nkv; ++j) {
-      // this tile's V; the next tile's K, or after the last tile the feature weights: Phi = X W^T is
-      // issued right behind the group's last P V, in the place the next tile's Q K^T would have
-      const bool last = (j + 1 == nkv);
-      const bool more = !last || lin;                         // a score-like product follows the P V
-      const int iv = base + 2 * j + 1, ik = last ? base + q.it_w : base + 2 * j + 2;
-      const uint32_t id_next = last ? ID_PHI : ID_QK;
-#pragma unroll
-      for (int g = 0; g < 2; ++g) {
-        uint64_t dv[8], dq[8], dk[8];
-        uint32_t ap[8];
-        {
-          const uint32_t xa = (last && layers == 2) ? q.sKV(base + q.it_h + g) : q.sQ(g);
-          const uint64_t v0 = mnmajor_desc(q.sKV(iv)), q0 = kmajor_desc(xa), k0 = kmajor_desc(q.sKV(ik));
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint64_t off = (uint64_t)(((kk / 4) * BOX_BYTES + (kk % 4) * 32) >> 4);
-            dv[kk] = v0 + (uint64_t)((kk * 2048) >> 4);
-            dq[kk] = q0 + off;
-            dk[kk] = k0 + off;
-            ap[kk] = q.tS(g) + kk * 8;
-          }
-        }
-        // P of this group and tile, and (first group only) the two ring tiles the block reads
-        if (!q.wait3(R::B_P + g, pb + j, g == 0, q.full_bar(iv), iv / KV_STAGES, g == 0 && more, q.full_bar(ik), ik / KV_STAGES))
-          return false;
-        if (last && layers == 2 && !q.wait1(q.full_bar(base + q.it_h + g), (base + q.it_h + g) / KV_STAGES)) return false;
-        tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) mma_ts(q.tO(g), ap[kk], dv[kk], ID_PV, (j > 0 || kk > 0) ? 1u : 0u);
-        if (more) {
-#pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), dq[kk], dk[kk], id_next, kk > 0 ? 1u : 0u);
-          tc_commit(q.bar(R::B_S + g));
-        } else {
-          tc_commit(q.bar(R::B_O + g));
-        }
-        if (last) {
-          tc_commit(q.bar(R::B_QF + g));             // nothing of this unit reads the group's Q tile any more
-          if (layers == 2) q.release(base + q.it_h + g);
-        }
-      }
-      q.release(iv);
-      if (more) q.release(ik);
+      if (nkv == 1 && !lin) tc_commit(q.bar(R::B_QF + g));
     }
   }
-  if (lin && nkv == 0) {
-    // no softmax tokens at all: the feature product opens the unit
-    if (!q.wait1(q.full_bar(base + q.it_w), (base + q.it_w) / KV_STAGES)) return false;
-    for (int g = 0; g < 2; ++g) {
-      // Phi = X W^T with X = Q (one layer) or the first-layer activations (two layers)
-      if (layers == 2 && !q.wait1(q.full_bar(base + q.it_h + g), (base + q.it_h + g) / KV_STAGES)) return false;
-      tc_fence_after();
-      issue_kmajor<D>(q.tS(g), kmajor_desc(layers == 2 ? q.sKV(base + q.it_h + g) : q.sQ(g)),
-                      kmajor_desc(q.sKV(base + q.it_w)), ID_PHI, false);
-      tc_commit(q.bar(R::B_S + g));
-      tc_commit(q.bar(R::B_QF + g));                 // nothing of this unit reads the group's Q tile any more
-      if (layers == 2) q.release(base + q.it_h + g);
-      if (g == 1) q.release(base + q.it_w);
+  for (int j = 0; j < nkv; ++j) {
+    const bool last = (j + 1 == nkv);
+    // as soon as the groups have read their score rows: the next tile's Q K^T, or Phi after the last tile
+    if (!last) {
+      const int ik = base + q.item_k(j + 1);
+      const uint64_t k0 = kmajor_desc(q.sKV(ik));
+#pragma unroll
+      for (int g = 0; g < 2; ++g) {
+        if (!q.wait2(R::B_SF + g, pb + j, g == 0, ik)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), dq[g][kk], k0 + kstep_kmajor(kk), ID_QK, kk > 0 ? 1u : 0u);
+        tc_commit(q.bar(R::B_S + g));
+        if (j + 2 == nkv && !lin) tc_commit(q.bar(R::B_QF + g));   // the unit's last read of the Q tile
+      }
+      q.release(ik);
+    } else if (lin) {
+      for (int g = 0; g < 2; ++g) {
+        if (!q.wait2(R::B_SF + g, pb + j, g == 0, base + q.it_w)) return false;
+        if (q.two && !q.wait_full(base + q.it_h + g)) return false;
+        tc_fence_after();
+        issue_phi(g);
+      }
     }
+  }
+  return true;
+}
+
+template <int D>
+__device__ __noinline__ bool q_accum_unit(const QParams& p, const QCtx& c, int u) {
+  using R = QRing<D>;
+  constexpr int F = D;
+  constexpr uint32_t ID_PV = make_idesc(128, D, 0, 1);        // O += P V and O += phi_q S  (V, S are MN-major)
+  const int nkv = p.nkv, lin = p.lin;
+  const R q(nkv, lin, p.layers, c);
+  const int base = u * q.n_items, pb = u * q.n_sp;            // first ring item / first barrier phase of the unit
+  uint64_t dp[2][8];                                          // the P tiles never move
+#pragma unroll
+  for (int g = 0; g < 2; ++g) {
+    const uint64_t p0 = kmajor_desc(q.sP(g));
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) dp[g][kk] = p0 + kstep_kmajor(kk);
+  }
+  for (int j = 0; j < nkv; ++j) {
+    const bool last = (j + 1 == nkv);
+    // as soon as P is in shared memory: O += P V
+    const int iv = base + q.item_v(j);
+    const uint64_t v0 = mnmajor_desc(q.sKV(iv));
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+      if (!q.wait2(R::B_P + g, pb + j, g == 0, iv)) return false;
+      tc_fence_after();
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) mma_ss(q.tO(g), dp[g][kk], v0 + kstep_mnmajor(kk), ID_PV, (j > 0 || kk > 0) ? 1u : 0u);
+      tc_commit(q.bar(R::B_PF + g));
+      if (last && !lin) tc_commit(q.bar(R::B_O + g));
+    }
+    q.release(iv);
   }
   if (lin) {
     const int is = base + q.it_st;
+    const uint64_t s0 = mnmajor_desc(q.sKV(is));
     for (int g = 0; g < 2; ++g) {
-      if (!q.wait3(R::B_P + g, pb + nkv, g == 0, q.full_bar(is), is / KV_STAGES, false, 0, 0)) return false;
+      if (!q.wait2(R::B_P + g, pb + nkv, g == 0, is)) return false;
       tc_fence_after();
-      // phi_q sits where P sits (bf16 over the score columns), S plays the part of a V tile
-      const uint64_t s0 = mnmajor_desc(q.sKV(is));
+      // phi_q sits where P sits, S plays the part of a V tile
 #pragma unroll
-      for (int kk = 0; kk < F / 16; ++kk)
-        mma_ts(q.tO(g), q.tS(g) + kk * 8, s0 + (uint64_t)((kk * 2048) >> 4), ID_PV, (nkv > 0 || kk > 0) ? 1u : 0u);
+      for (int kk = 0; kk < F / 16; ++kk) mma_ss(q.tO(g), dp[g][kk], s0 + kstep_mnmajor(kk), ID_PV, (nkv > 0 || kk > 0) ? 1u : 0u);
+      tc_commit(q.bar(R::B_PF + g));
       tc_commit(q.bar(R::B_O + g));
       if (g == 1) q.release(is);
     }
@@ -313,16 +374,27 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
   const int r = (warp & 3) * 32 + lane;             // row inside the group's 128-row tile
   const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
   const uint32_t tSg = q.tS(g) + lane_off, tOg = q.tO(g) + lane_off;
+  uint8_t* sPg = smem + L::P_OFF + g * L::PTILE;    // this group's P / phi_q / output staging tile
   const int pb = u * q.n_sp;
   float m_ref = 0.f, m_true = -INFINITY, l = 0.f;
   uint32_t x[32];
+
+  // The P buffer may be written once the product that read its previous contents has completed; the very
+  // first use only has to wait for this warp's output store of the previous unit to have been read out.
+  auto p_buffer_free = [&](int use) -> bool {       // use: running index of the buffer's uses
+    if (lane == 0) tma_store_wait_read();
+    if (use == 0) { __syncwarp(); return true; }
+    return q.wait(R::B_PF + g, use - 1);
+  };
 
   for (int j = 0; j < nkv; ++j) {
     if (!q.wait(R::B_S + g, pb + j)) return false;
     tc_fence_after();
     uint32_t sv[128];                               // this thread's row of the 128 x 128 score tile
     tmem_ld128_sync(tSg, sv);
-    const int valid = n_s - j * 128;              // keys of this tile that exist (>= 128: all)
+    tc_fence_before();
+    mbar_arrive(q.bar(R::B_SF + g));                // the score columns may be overwritten
+    const int valid = n_s - j * 128;                // keys of this tile that exist (>= 128: all)
     if (valid < 128) {
 #pragma unroll
       for (int i = 0; i < 128; ++i) sv[i] = (i < valid) ? sv[i] : 0xff800000u;   // -inf: exp2 gives 0
@@ -338,11 +410,11 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
     mx *= scale_log2;
     m_true = fmaxf(m_true, mx);
     // The reference maximum only moves when the row maximum grew by more than 2^8; then O and l
-    // are rescaled (after P is out of the registers; the MMA that adds P V waits for this thread).
+    // are rescaled (once the previous tile's P V has completed, before this tile's P is handed over).
     const bool need = (j > 0) && (mx > m_ref + RESCALE_THRESHOLD);
     const float resc = need ? ex2(m_ref - mx) : 1.f;
     if (j == 0 || need) m_ref = mx;
-    // P = exp2(s * scale_log2 - m_ref) as bf16, written over the first 64 columns of S
+    // P = exp2(s * scale_log2 - m_ref) as bf16 into the group's P tile in shared memory
     const float neg_m = -m_ref;
     // packed fp32x2 arithmetic halves the instruction count of the scaling and of the row sum
     const float2 scale2 = make_float2(scale_log2, scale_log2), negm2 = make_float2(neg_m, neg_m);
@@ -361,11 +433,13 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
         pw[2 * i] = pack_bf16(pa.x, pa.y);
         pw[2 * i + 1] = pack_bf16(pc.x, pc.y);
       }
-      tmem_st16(tSg + cc * 16, pw);
+      if (cc == 0 && !p_buffer_free(pb + j)) return false;   // the previous tile's P V has read the buffer
+      store_row_chunk(sPg, r, cc * 32, pw);
     }
     l = l * resc + ((la.x + la.y) + (lb.x + lb.y));
     if (__any_sync(0xffffffffu, need)) {
-      // O += P V of the previous tile has completed (its commit precedes this tile's S barrier)
+      // the previous tile's P V has completed (waited for above) and this tile's has not been released yet
+      tc_fence_after();
 #pragma unroll
       for (int cc = 0; cc < D / 32; ++cc) {
         tmem_ld32(tOg + cc * 32, x);
@@ -374,9 +448,10 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
         for (int i = 0; i < 32; ++i) x[i] = __float_as_uint(__uint_as_float(x[i]) * resc);
         tmem_st32(tOg + cc * 32, x);
       }
+      tmem_st_wait();
+      tc_fence_before();
     }
-    tmem_st_wait();
-    tc_fence_before();
+    fence_proxy_async();
     mbar_arrive(q.bar(R::B_P + g));
   }
 
@@ -393,17 +468,26 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
     const float2* zrow = reinterpret_cast<const float2*>(p.z + (size_t)bh * F);
     if (!q.wait(R::B_S + g, pb + nkv)) return false;
     tc_fence_after();
+    uint32_t ph[F];                                  // this thread's row of Phi: read at once, columns released
     float dl0 = 0.f, dl1 = 0.f;
     const bool two_parts = (p.P == 2);
 #pragma unroll
     for (int cc = 0; cc < F / 32; ++cc) {
       tmem_ld32(tSg + cc * 32, x);
       tmem_ld_wait(x);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) ph[cc * 32 + i] = x[i];
+    }
+    tc_fence_before();
+    mbar_arrive(q.bar(R::B_SF + g));                 // the next unit's first Q K^T may overwrite the columns
+    if (!p_buffer_free(pb + nkv)) return false;      // the last tile's P V has read the buffer
+#pragma unroll
+    for (int cc = 0; cc < F / 32; ++cc) {
       const bool squared = two_parts && (cc * 32 >= F / 2);
       uint32_t wd[16];
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
-        float a0 = fmaxf(__uint_as_float(x[2 * i]), 0.f), a1 = fmaxf(__uint_as_float(x[2 * i + 1]), 0.f);
+        float a0 = fmaxf(__uint_as_float(ph[cc * 32 + 2 * i]), 0.f), a1 = fmaxf(__uint_as_float(ph[cc * 32 + 2 * i + 1]), 0.f);
         if (squared) { a0 *= a0; a1 *= a1; }
         wd[i] = pack_bf16(a0 * lam, a1 * lam);
         // the denominator uses the very bf16 values the MMA multiplies with S
@@ -411,11 +495,10 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
         dl0 = fmaf(__uint_as_float(wd[i] << 16), zz.x, dl0);
         dl1 = fmaf(__uint_as_float(wd[i] & 0xffff0000u), zz.y, dl1);
       }
-      tmem_st16(tSg + cc * 16, wd);                  // over Phi columns this thread has already read
+      store_row_chunk(sPg, r, cc * 32, wd);          // phi_q takes P's place as the A operand
     }
     const float dl = dl0 + dl1;
-    tmem_st_wait();
-    tc_fence_before();
+    fence_proxy_async();
     mbar_arrive(q.bar(R::B_P + g));
     den = l + dl;
     den_l_out = dl / lam;
@@ -423,33 +506,26 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
   if (!q.wait(R::B_O + g, u)) return false;
   tc_fence_after();
   const float inv = 1.f / den;
-  // Each warp stages its 32 rows, 64 columns at a time, in a buffer of its own and hands them to a
-  // TMA store (rows past N are clipped by the tensor map); no other warp is waited for.
-  uint8_t* stg = smem + L::OUT_OFF + warp * L::OUT_WARP;
+  // The output rows are staged in the group's P tile (the product that read it has completed with the O
+  // barrier); each warp stores its own 32 rows (rows past N are clipped by the tensor map).
   const int wrow0 = row - lane;
 #pragma unroll
-  for (int half = 0; half < D / 64; ++half) {
-    uint32_t wd[32];
+  for (int cc = 0; cc < D / 32; ++cc) {
+    tmem_ld32(tOg + cc * 32, x);
+    tmem_ld_wait(x);
+    uint32_t wd[16];
 #pragma unroll
-    for (int cc = 0; cc < 2; ++cc) {
-      tmem_ld32(tOg + half * 64 + cc * 32, x);
-      tmem_ld_wait(x);
+    for (int i = 0; i < 16; ++i)
+      wd[i] = pack_bf16(__uint_as_float(x[2 * i]) * inv, __uint_as_float(x[2 * i + 1]) * inv);
+    store_row_chunk(sPg, r, cc * 32, wd);
+  }
+  fence_proxy_async();
+  __syncwarp();
+  if (lane == 0 && wrow0 < p.N) {
 #pragma unroll
-      for (int i = 0; i < 16; ++i)
-        wd[cc * 16 + i] = pack_bf16(__uint_as_float(x[2 * i]) * inv, __uint_as_float(x[2 * i + 1]) * inv);
-    }
-    if (lane == 0) tma_store_wait_read();            // the buffer's previous store has been read out
-    __syncwarp();
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-      *reinterpret_cast<uint4*>(stg + swz128_chunk_offset(lane, i)) =
-          make_uint4(wd[4 * i], wd[4 * i + 1], wd[4 * i + 2], wd[4 * i + 3]);
-    fence_proxy_async();
-    __syncwarp();
-    if (lane == 0 && wrow0 < p.N) {
-      tma_store_3d(tmO, smem_u32(stg), half * 64, wrow0, bh);
-      tma_store_commit();
-    }
+    for (int b = 0; b < D / 64; ++b)
+      tma_store_3d(tmO, smem_u32(sPg) + b * BOX_BYTES + (warp & 3) * 32 * 128, b * 64, wrow0, bh);
+    tma_store_commit();
   }
   if (p.aux != nullptr && row < p.N) {
     const float ln2 = 0.6931471805599453f;
@@ -491,7 +567,8 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     mbar_init(bar(R::B_Q0), 1); mbar_init(bar(R::B_Q0 + 1), 1);
     for (int s = 0; s < KV_STAGES; ++s) { mbar_init(bar(R::B_FULL + s), 1); mbar_init(bar(R::B_EMPTY + s), 1); }
     for (int g = 0; g < 2; ++g) {
-      mbar_init(bar(R::B_S + g), 1); mbar_init(bar(R::B_P + g), 128); mbar_init(bar(R::B_O + g), 1); mbar_init(bar(R::B_QF + g), 1);
+      mbar_init(bar(R::B_S + g), 1); mbar_init(bar(R::B_SF + g), 128); mbar_init(bar(R::B_P + g), 128);
+      mbar_init(bar(R::B_PF + g), 1); mbar_init(bar(R::B_O + g), 1); mbar_init(bar(R::B_QF + g), 1);
     }
     fence_barrier_init();
     fence_proxy_async();
@@ -510,7 +587,13 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   } else if (warp == 9) {
     if ((threadIdx.x & 31) == 0) {
       for (int u = 0; u < n_mine; ++u)
-        if (!q_mma_unit<D>(p, c, u)) break;
+        if (!q_score_unit<D>(p, c, u)) break;
+    }
+    __syncwarp();
+  } else if (warp == 10) {
+    if ((threadIdx.x & 31) == 0) {
+      for (int u = 0; u < n_mine; ++u)
+        if (!q_accum_unit<D>(p, c, u)) break;
     }
     __syncwarp();
   } else {
