@@ -421,3 +421,26 @@ def test_host_entry_point_pipelined_over_runs_of_heads():
         assert torch.equal(out_host, ref.view(torch.int16).cpu())
         S, z = op.linear_state()
         assert torch.equal(S, S_ref) and torch.equal(z, z_ref)
+
+
+# More (batch, head) pairs than SMs, so that a persistent CTA walks over several units, with key loops of
+# one, two and three tiles and with / without the linear tail: the hand-overs at unit boundaries (Q tile
+# release, score columns, P tile, output accumulator) all happen with barrier phases that run on.
+MANY_UNITS = {
+    "one_key_tile_softmax_only": W.Workload("u1", B=2, H=80, d=128, F=128, grid=(1, 5, 7), block=(1, 5, 7), rate=1, seed=31),
+    "two_key_tiles_softmax_only": W.Workload("u2", B=2, H=80, d=128, F=128, grid=(1, 10, 20), block=(1, 10, 20), rate=1, seed=32),
+    "one_key_tile_hybrid": W.Workload("u3", B=2, H=80, d=128, F=128, grid=(1, 10, 30), block=(1, 5, 6), rate=3, seed=33),
+    "three_key_tiles_hybrid_d64": W.Workload("u4", B=3, H=60, d=64, F=64, grid=(2, 12, 25), block=(1, 4, 5), rate=2, seed=34,
+                                             rms_norm_qk=False),
+    "no_key_tile_linear_only": W.Workload("u5", B=2, H=80, d=128, F=128, grid=(1, 10, 30), block=(1, 5, 6), rate=0, seed=35),
+}
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("name", sorted(MANY_UNITS))
+def test_many_units_per_cta(mode, name):
+    wl = MANY_UNITS[name]
+    gain = balanced_gain(wl, mode)
+    got, got_aux, ref, ref_aux, ex = _run(wl, FULL_PATH, mode, gain)
+    assert_parity(got, ref, name, strict=False)
+    _check_aux(got_aux, ref_aux, wl, ex["n_softmax"])
