@@ -338,6 +338,12 @@ TWO_LAYER = {
                                   rate=0, seed=33, layers=2),
     "two_layer_chunks": W.Workload("two_layer_chunks", B=1, H=1, d=128, F=128, grid=(8, 30, 52), block=(1, 6, 8),
                                    rate=8, seed=34, layers=2),
+    # more (batch, head) pairs than SMs: several units per persistent CTA, with the two first-layer tiles,
+    # the weights and the last V tile competing for the three ring slots at every unit's end
+    "two_layer_many_units": W.Workload("two_layer_many_units", B=2, H=80, d=128, F=128, grid=(1, 10, 30), block=(1, 5, 6),
+                                       rate=3, seed=35, layers=2),
+    "two_layer_many_units_rate0": W.Workload("two_layer_many_units_rate0", B=2, H=80, d=64, F=64, grid=(1, 10, 30),
+                                             block=(1, 5, 6), rate=0, seed=36, layers=2, rms_norm_qk=False),
 }
 
 
