@@ -47,7 +47,7 @@ typedef struct as_hybrid_attn_s* as_hybrid_attn_t;   /* opaque, library-owned */
 typedef enum {
   AS_OK = 0,
   AS_ERR_INVALID_ARG = 1,     /* NULL pointer, bad shape, misaligned buffer, inconsistent sizes   */
-  AS_ERR_UNSUPPORTED = 2,     /* valid request that this build has no kernel for                   */
+  AS_ERR_UNSUPPORTED = 2,     /* valid request the library has no kernel for                      */
   AS_ERR_ARCH = 3,            /* current device is not compute capability 10.x                      */
   AS_ERR_ALLOC = 4,           /* host or device allocation failed in create                        */
   AS_ERR_WORKSPACE = 5,       /* workspace NULL, misaligned or smaller than workspace_bytes         */

@@ -51,7 +51,7 @@ as_status_t validate(const as_hybrid_attn_desc_t* d) {
   if (!(d->softmax_scale >= 0.f) || !std::isfinite(d->softmax_scale)) return AS_ERR_INVALID_ARG;
   if (d->phi_dim <= 0 || d->poly_degree <= 0 || d->phi_layers <= 0) return AS_ERR_INVALID_ARG;
   if (d->phi_dim % d->poly_degree != 0) return AS_ERR_INVALID_ARG;
-  // what this build has kernels for
+  // what the library has kernels for
   if (d->d != 64 && d->d != 128) return AS_ERR_UNSUPPORTED;
   if (d->phi_dim != d->d) return AS_ERR_UNSUPPORTED;
   if (d->phi_layers > 2 || d->poly_degree > 2 || d->phi_act != AS_ACT_RELU) return AS_ERR_UNSUPPORTED;
