@@ -28,7 +28,7 @@ METRIC = "hybrid-attn fwd tokens/s per layer at N=32760 (12x128 heads); % of bf1
 
 # DRAM bytes of one Q-pass launch at the wan81 workload (dram__bytes_read.sum + dram__bytes_write.sum
 # from the ncu capture summarised in profiles/); None until a capture exists.
-QPASS_DRAM_TRAFFIC_BYTES = {"wan81": 126722304 + 63252480}
+QPASS_DRAM_TRAFFIC_BYTES = {"wan81": 126750464 + 63403008}
 
 
 def _peaks():

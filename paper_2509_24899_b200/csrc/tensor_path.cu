@@ -7,7 +7,8 @@
 //                          z    += row sums of the bf16 features (registers)
 //     softmax-token rows of the K / V tiles are copied from shared memory to the compact K_S / V_S.
 //   Q pass  (steps: softmax branch, phi_q projection, linear apply, merge)
-//     persistent, one CTA per SM; per unit of 2 x 128 query rows a flash-style loop over 128-key tiles
+//     persistent, one CTA per SM (units left over after the full rounds are split into 128-row halves
+//     over twice as many CTAs); per unit of 2 x 128 query rows a flash-style loop over 128-key tiles
 //     of K_S / V_S:        S = Q K_S^T -> TMEM; the softmax threads (one per row) read their row and
 //                          release the score columns at once, so the next tile's Q K_S^T runs under the
 //                          exponentials; running max / sum per row; P = exp2(.) as bf16 -> shared memory,
@@ -38,6 +39,8 @@ struct QParams {
   int N, n_s, nkv, lin, stab_mode, P, H;
   int layers;                // depth of the feature map: with 2, tmH holds relu(q W_1^T) and tmW is W_2
   int nx, n_units;           // 256-row units per (batch, head); units over all (batch, head) pairs
+  int n_rounds;              // rounds in which every CTA has a unit (n_units / gridDim.x)
+  int split_last;            // 1: the units left over after those rounds are cut in two 128-row halves, one per CTA
   float scale_log2;          // softmax scale * log2(e)
   const float* z;            // [B*H][F]
   float* aux;                // [B*H][N][3] or nullptr
@@ -119,6 +122,26 @@ struct QCtx {
   WaitCtx wc;
 };
 
+// Unit u of this CTA: which 256-row unit, which row it starts at, and how many of the two 128-row groups
+// work on it.  In the rounds every CTA takes part in, CTA c has unit c + u * gridDim.x.  What is left
+// over afterwards would keep less than half of the SMs busy for a whole unit's time; a single group, which
+// has the tensor and XU pipes to itself, needs little more than half of that, so the left-over units are
+// cut into their two 128-row halves and spread over twice as many CTAs.
+struct QUnit { int w, row0, ng; };
+AS_DEV QUnit q_unit(const QParams& p, int u) {
+  const int c = (int)blockIdx.x, n = (int)gridDim.x;
+  if (u < p.n_rounds) { const int w = c + u * n; return QUnit{w, (w % p.nx) * 256, 2}; }
+  if (p.split_last) { const int w = p.n_rounds * n + (c >> 1); return QUnit{w, (w % p.nx) * 256 + (c & 1) * 128, 1}; }
+  const int w = p.n_rounds * n + c;
+  return QUnit{w, (w % p.nx) * 256, 2};
+}
+// number of units CTA c walks over
+AS_DEV int q_units_of_cta(const QParams& p) {
+  const int left = p.n_units - p.n_rounds * (int)gridDim.x;
+  const int extra = p.split_last ? ((int)blockIdx.x < 2 * left) : ((int)blockIdx.x < left);
+  return p.n_rounds + (extra ? 1 : 0);
+}
+
 template <int D>
 struct QRing {
   using L = QLayout<D>;
@@ -179,14 +202,14 @@ __device__ __noinline__ bool q_produce_unit(const QParams& p, const QCtx& c, con
   const int nkv = p.nkv;
   const R q(nkv, p.lin, p.layers, c);
   const int lane = threadIdx.x & 31;
-  const int w = (int)blockIdx.x + u * (int)gridDim.x;
-  const int bh = w / p.nx, h = bh % p.H, row0 = (w % p.nx) * 256;
+  const QUnit un = q_unit(p, u);
+  const int bh = un.w / p.nx, h = bh % p.H, row0 = un.row0;
   const int base = u * q.n_items;
   const int n_stream = nkv > 0 ? 2 * nkv - 1 : 0;     // K_0, then K_{j+1}, V_j alternating
   const int q_at = nkv > 0 ? 1 : 0;                   // the Q tiles are requested right after the unit's first K tile
   for (int it = 0; it < q.n_items; ++it) {
     if (it == q_at) {
-      for (int g = 0; g < 2; ++g) {
+      for (int g = 0; g < un.ng; ++g) {
         // the previous unit's last product that reads this Q buffer has completed
         if (u > 0 && !q.wait(R::B_QF + g, u - 1)) return false;
         if (lane == 0) {
@@ -237,6 +260,7 @@ __device__ __noinline__ bool q_score_unit(const QParams& p, const QCtx& c, int u
   const int nkv = p.nkv, lin = p.lin;
   const R q(nkv, lin, p.layers, c);
   const int base = u * q.n_items, pb = u * q.n_sp;            // first ring item / first barrier phase of the unit
+  const int ng = q_unit(p, u).ng;                             // groups at work on this unit (the last one of a group: ng - 1)
   uint64_t dq[2][8];                                          // the Q tiles do not move within a unit
 #pragma unroll
   for (int g = 0; g < 2; ++g) {
@@ -258,11 +282,15 @@ __device__ __noinline__ bool q_score_unit(const QParams& p, const QCtx& c, int u
     tc_commit(q.bar(R::B_S + g));
     tc_commit(q.bar(R::B_QF + g));                   // nothing of this unit reads the group's Q tile any more
     if (q.two) q.release(base + q.it_h + g);
-    if (g == 1) q.release(base + q.it_w);
+    if (g == ng - 1) {
+      // a lone group: the other group's first-layer tile was loaded all the same and only has to be let go
+      if (q.two && ng == 1) { q.wait_full(base + q.it_h + 1); q.release(base + q.it_h + 1); }
+      q.release(base + q.it_w);
+    }
   };
   // The first product of a unit overwrites score columns the previous unit's threads read last: wait for
   // that read (the last S-free phase of the previous unit) together with the Q tile.
-  for (int g = 0; g < 2; ++g) {
+  for (int g = 0; g < ng; ++g) {
     if (u > 0 && !q.wait1(R::B_SF + g, pb - 1)) return false;
     if (nkv == 0) {
       if (!q.wait1(R::B_Q0 + g, u)) return false;
@@ -280,7 +308,7 @@ __device__ __noinline__ bool q_score_unit(const QParams& p, const QCtx& c, int u
 #pragma unroll
       for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), dq[g][kk], k0 + kstep_kmajor(kk), ID_QK, kk > 0 ? 1u : 0u);
       tc_commit(q.bar(R::B_S + g));
-      if (g == 1) q.release(base);
+      if (g == ng - 1) q.release(base);
       if (nkv == 1 && !lin) tc_commit(q.bar(R::B_QF + g));
     }
   }
@@ -292,6 +320,7 @@ __device__ __noinline__ bool q_score_unit(const QParams& p, const QCtx& c, int u
       const uint64_t k0 = kmajor_desc(q.sKV(ik));
 #pragma unroll
       for (int g = 0; g < 2; ++g) {
+        if (g >= ng) break;
         if (!q.wait2(R::B_SF + g, pb + j, g == 0, ik)) return false;
         tc_fence_after();
 #pragma unroll
@@ -301,7 +330,7 @@ __device__ __noinline__ bool q_score_unit(const QParams& p, const QCtx& c, int u
       }
       q.release(ik);
     } else if (lin) {
-      for (int g = 0; g < 2; ++g) {
+      for (int g = 0; g < ng; ++g) {
         if (!q.wait2(R::B_SF + g, pb + j, g == 0, base + q.it_w)) return false;
         if (q.two && !q.wait_full(base + q.it_h + g)) return false;
         tc_fence_after();
@@ -320,6 +349,7 @@ __device__ __noinline__ bool q_accum_unit(const QParams& p, const QCtx& c, int u
   const int nkv = p.nkv, lin = p.lin;
   const R q(nkv, lin, p.layers, c);
   const int base = u * q.n_items, pb = u * q.n_sp;            // first ring item / first barrier phase of the unit
+  const int ng = q_unit(p, u).ng;
   uint64_t dp[2][8];                                          // the P tiles never move
 #pragma unroll
   for (int g = 0; g < 2; ++g) {
@@ -334,6 +364,7 @@ __device__ __noinline__ bool q_accum_unit(const QParams& p, const QCtx& c, int u
     const uint64_t v0 = mnmajor_desc(q.sKV(iv));
 #pragma unroll
     for (int g = 0; g < 2; ++g) {
+      if (g >= ng) break;
       if (!q.wait2(R::B_P + g, pb + j, g == 0, iv)) return false;
       tc_fence_after();
 #pragma unroll
@@ -346,7 +377,7 @@ __device__ __noinline__ bool q_accum_unit(const QParams& p, const QCtx& c, int u
   if (lin) {
     const int is = base + q.it_st;
     const uint64_t s0 = mnmajor_desc(q.sKV(is));
-    for (int g = 0; g < 2; ++g) {
+    for (int g = 0; g < ng; ++g) {
       if (!q.wait2(R::B_P + g, pb + nkv, g == 0, is)) return false;
       tc_fence_after();
       // phi_q sits where P sits, S plays the part of a V tile
@@ -354,7 +385,7 @@ __device__ __noinline__ bool q_accum_unit(const QParams& p, const QCtx& c, int u
       for (int kk = 0; kk < F / 16; ++kk) mma_ss(q.tO(g), dp[g][kk], s0 + kstep_mnmajor(kk), ID_PV, (nkv > 0 || kk > 0) ? 1u : 0u);
       tc_commit(q.bar(R::B_PF + g));
       tc_commit(q.bar(R::B_O + g));
-      if (g == 1) q.release(is);
+      if (g == ng - 1) q.release(is);
     }
   }
   return true;
@@ -455,9 +486,9 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
     mbar_arrive(q.bar(R::B_P + g));
   }
 
-  const int w = (int)blockIdx.x + u * (int)gridDim.x;
-  const int bh = w / p.nx;
-  const int row = (w % p.nx) * 256 + g * 128 + r;
+  const QUnit un = q_unit(p, u);
+  const int bh = un.w / p.nx;
+  const int row = un.row0 + g * 128 + r;
   float den = l, den_l_out = 0.f;
   if (p.lin) {
     // per-row factor applied to phi_q so that the linear branch lands on the scale of O and l
@@ -578,7 +609,7 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   __syncthreads();
   tc_fence_after();
   const QCtx c{sbase, *tmem_slot, WaitCtx{p.status, abort_flag}};
-  const int n_mine = (p.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // units of this CTA
+  const int n_mine = q_units_of_cta(p);               // units of this CTA
 
   if (warp == 8) {
     if ((threadIdx.x & 31) == 0) { tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmO); }
@@ -597,7 +628,9 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     }
     __syncwarp();
   } else {
-    for (int u = 0; u < n_mine; ++u)
+    // a unit worked on by one group only (a left-over half) is the CTA's last one: group 1 stops before it
+    const int n_grp = (n_mine > p.n_rounds && p.split_last && warp >= 4) ? p.n_rounds : n_mine;
+    for (int u = 0; u < n_grp; ++u)
       if (!q_softmax_unit<D>(p, c, &tmO, smem, u)) break;
     if ((threadIdx.x & 31) == 0) tma_store_wait_all();   // this warp's output stores have completed
   }
@@ -1093,6 +1126,10 @@ cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st) {
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
     return cudaErrorInvalidValue;
   dim3 grid(p.n_units < sms ? p.n_units : sms, 1, 1);
+  p.n_rounds = p.n_units / (int)grid.x;
+  const int left = p.n_units - p.n_rounds * (int)grid.x;
+  // left-over units as 128-row halves when twice their number still fits the grid
+  p.split_last = (left > 0 && 2 * left <= (int)grid.x) ? 1 : 0;
   if (a.d == 128) qpass_kernel<128><<<grid, Q_THREADS, QLayout<128>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmH, tmO, p);
   else qpass_kernel<64><<<grid, Q_THREADS, QLayout<64>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmH, tmO, p);
   return cudaGetLastError();
