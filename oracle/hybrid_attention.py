@@ -22,9 +22,10 @@ Readings taken where the paper is silent (each is restated next to the code):
   multiplied by exp(-c_i)); STAB_EXACT multiplies the linear terms by exp(-c_i), which
   makes the result independent of c_i (weights exp(s_ij) next to phi_q.phi_k).
 * The embedding network is `layers` linear maps, each followed by ReLU (also the last
-  one, so that phi >= 0 as the paper requires).  The activation choice itself is not
-  fixed by the paper: parity unpinned for that choice (the pins below fix everything
-  else about phi).
+  one, so that phi >= 0 as the paper requires), each with an optional bias added before
+  the ReLU.  The activation choice itself is not fixed by the paper: parity unpinned for
+  that choice (the pins fix everything else about phi: layer order, the inner ReLU, the
+  bias placement and the powers are checked against hand-worked values).
 * Rate 1 means every token is a softmax token; rate 0 means none is.
 * With a spatial block (t, h, w) on the latent grid the 1-D rule is applied to the
   raster index inside each (clipped) block; with one block covering the whole grid
@@ -76,21 +77,23 @@ def softmax_token_mask(grid, block, rate):
 # --------------------------------------------------------------------------------------
 # Feature map ("Characterization of phi")
 # --------------------------------------------------------------------------------------
-def phi_features(x, weights, degree=2, biases=None):
+def phi_features(x, weights, degree=2):
     """phi(x) for x[..., d] with one head's embedding network.
 
-    weights: list of matrices, weights[l] has shape [out_l, in_l]; the network is
-             a_0 = x, a_{l+1} = ReLU(weights[l] @ a_l (+ biases[l])).
+    weights: one matrix, or a list with one entry per layer; an entry is a matrix W_l of shape
+             [out_l, in_l] or a pair (W_l, b_l) with a bias vector b_l [out_l].  The network is
+             a_0 = x, a_{l+1} = ReLU(W_l a_l + b_l)  (b_l = 0 when no bias is given).
     The last activation [..., F] is split into `degree` = P contiguous equal parts;
     part p (1-indexed) is raised elementwise to the power p; parts are concatenated.
     """
     a = np.asarray(x, dtype=np.float64)
     if isinstance(weights, np.ndarray):
         weights = [weights]
-    for l, W in enumerate(weights):
+    for l, layer in enumerate(weights):
+        W, b = layer if isinstance(layer, tuple) else (layer, None)
         a = a @ np.asarray(W, dtype=np.float64).T
-        if biases is not None and biases[l] is not None:
-            a = a + np.asarray(biases[l], dtype=np.float64)
+        if b is not None:
+            a = a + np.asarray(b, dtype=np.float64)
         a = np.maximum(a, 0.0)
     F = a.shape[-1]
     P = int(degree)

@@ -203,15 +203,45 @@ def test_exact_mode_is_the_unstabilised_ratio_and_paper_mode_depends_on_c():
     np.testing.assert_allclose(ratio_p, ratio_e * np.exp(aux[:, 0]), rtol=1e-10)
 
 
-def test_phi_is_nonnegative_and_two_layer_shape():
+def _phi_cases():
+    with open(GOLDEN) as f:
+        return json.load(f)["phi_cases"]
+
+
+def _layers(case):
+    return [(np.array(l["W"], float), np.array(l["b"], float)) if "b" in l else np.array(l["W"], float)
+            for l in case["layers"]]
+
+
+@pytest.mark.parametrize("case", _phi_cases(), ids=lambda c: c["name"])
+def test_feature_map_hand_worked_values(case, oracle=O):
+    """Multi-layer embedding network, bias placement and power order against values worked by hand."""
+    f = oracle.phi_features(np.array(case["x"], float), _layers(case), degree=case["degree"])
+    np.testing.assert_allclose(f, np.array(case["phi"], float), rtol=1e-14, atol=1e-14)
+
+
+def test_phi_is_nonnegative_and_shapes():
     rng = np.random.default_rng(7)
     x = rng.standard_normal((5, 4))
     w1, w2 = rng.standard_normal((8, 4)), rng.standard_normal((6, 8))
-    f = O.phi_features(x, [w1, w2], degree=3)
+    f = O.phi_features(x, [w1, (w2, rng.standard_normal(6))], degree=3)
     assert f.shape == (5, 6) and (f >= 0).all()
-    a = np.maximum(np.maximum(x @ w1.T, 0) @ w2.T, 0)
-    np.testing.assert_allclose(f[:, 4:], a[:, 4:] ** 3)
-    np.testing.assert_allclose(f[:, :2], a[:, :2])
+
+
+@pytest.mark.parametrize("mode", [O.STAB_PAPER, O.STAB_EXACT])
+def test_two_layer_operator_reduces_to_one_layer_when_the_second_is_the_identity(mode):
+    # ReLU is idempotent, so [W, I] must give exactly what [W] gives, through the whole operator.
+    rng = np.random.default_rng(17)
+    q, k, v, wq, wk, mask = _rand_case(rng, N=24, d=6, F=8, R=3)
+    eye = np.eye(8)
+    y1, aux1 = O.hybrid_attention_head(q, k, v, wq, wk, mask, None, mode)
+    y2, aux2 = O.hybrid_attention_head(q, k, v, [wq, eye], [wk, eye], mask, None, mode)
+    np.testing.assert_allclose(y2, y1, rtol=1e-13)
+    np.testing.assert_allclose(aux2, aux1, rtol=1e-13)
+    S1, z1 = O.linear_state(k, v, wk, mask)
+    S2, z2 = O.linear_state(k, v, [(wk, np.zeros(8)), eye], mask)
+    np.testing.assert_allclose(S2, S1, rtol=1e-13)
+    np.testing.assert_allclose(z2, z1, rtol=1e-13)
 
 
 def test_rows_argument_selects_rows():
@@ -253,6 +283,12 @@ def _mutants():
         "scale_missing": ("s = (qb @ k_s.T) * scale ", "s = (qb @ k_s.T) "),
         "lambda_inverted": ("lam = np.exp(-c)", "lam = np.exp(c)"),
         "S_transposed_use": ("num += lam[:, None] * (fq @ S)", "num += lam[:, None] * (fq @ S.T)"),
+        "layers_in_reverse_order": ("for l, layer in enumerate(weights):", "for l, layer in enumerate(list(weights)[::-1]):"),
+        "inner_relu_missing": ("a = np.maximum(a, 0.0)", "a = np.maximum(a, 0.0) if l == len(weights) - 1 else a"),
+        "bias_dropped": ("a = a + np.asarray(b, dtype=np.float64)", "a = a"),
+        "bias_after_relu": ("a = a + np.asarray(b, dtype=np.float64)\n        a = np.maximum(a, 0.0)",
+                            "a = np.maximum(a, 0.0)\n            a = a + np.asarray(b, dtype=np.float64)\n"
+                            "        a = a if b is not None else np.maximum(a, 0.0)"),
     }
     for name, (old, new) in edits.items():
         assert src.count(old) == 1, name
@@ -268,6 +304,11 @@ def test_planted_mistakes_are_caught(name, mutant):
     for case in _golden_cases():
         try:
             test_hand_worked_values(case, "factorised", oracle=mutant)
+        except (AssertionError, ValueError):
+            failures += 1
+    for case in _phi_cases():
+        try:
+            test_feature_map_hand_worked_values(case, oracle=mutant)
         except (AssertionError, ValueError):
             failures += 1
     try:
