@@ -56,10 +56,15 @@ class HybridAttention:
     def softmax_indices(self):
         return binding.as_hybrid_attn_softmax_tokens(self._h)[1]
 
-    def forward(self, q, k, v, wq=None, wk=None, out=None, aux=None, stream=None, wq2=None, wk2=None):
+    def forward(self, q, k, v, wq=None, wk=None, out=None, aux=None, stream=None, wq2=None, wk2=None,
+                workspace=None):
+        """`workspace` (optional): a caller-owned uint8 CUDA tensor of at least `workspace_bytes`, 256-byte
+        aligned; it becomes the handle's workspace for `linear_state` as well."""
         import torch
         if out is None:
             out = torch.empty_like(q)
+        if workspace is not None:
+            self._ws = workspace
         ws = self.workspace()
         st = torch.cuda.current_stream() if stream is None else stream
         binding.as_hybrid_attn_forward(

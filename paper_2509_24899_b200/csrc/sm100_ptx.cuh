@@ -205,6 +205,15 @@ AS_DEV uint32_t pack_bf16(float lo, float hi) {
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
+// a += low half of w, b += high half of w, the halves read as bf16 (mixed-precision add of sm_100)
+AS_DEV void add_bf16x2(float& a, float& b, uint32_t w) {
+  asm("{\n\t.reg .b16 lo, hi;\n\t"
+      "mov.b32 {lo, hi}, %2;\n\t"
+      "add.rn.f32.bf16 %0, lo, %0;\n\t"
+      "add.rn.f32.bf16 %1, hi, %1;\n\t}"
+      : "+f"(a), "+f"(b)
+      : "r"(w));
+}
 // three-input maximum (one instruction on sm_100)
 AS_DEV float fmax3(float a, float b, float c) {
   float d;

@@ -1,36 +1,22 @@
-// Tensor-core path of the hybrid attention forward for sm_100a (AS_PATH_TENSOR).
+// Q pass of the hybrid attention forward on the tensor cores of sm_100a: softmax branch, phi_q
+// projection, linear apply and merge, fused in one persistent kernel.
 //
-//   K pass  (steps: phi_k projection, linear state, softmax gather)
-//     per 128-token tile:  Phi^T = W_k K^T        (tcgen05.mma, smem x smem -> TMEM, lanes = features)
-//                          phi   = poly(relu(.)), zeroed for softmax tokens, bf16 back into TMEM
-//                          S    += phi^T-tile V   (tcgen05.mma, TMEM x smem -> TMEM accumulator)
-//                          z    += row sums of the bf16 features (registers)
-//     softmax-token rows of the K / V tiles are copied from shared memory to the compact K_S / V_S.
-//   Q pass  (steps: softmax branch, phi_q projection, linear apply, merge)
-//     persistent, one CTA per SM (units left over after the full rounds are split into 128-row halves
-//     over twice as many CTAs); per unit of 2 x 128 query rows a flash-style loop over 128-key tiles
-//     of K_S / V_S:        S = Q K_S^T -> TMEM; the softmax threads (one per row) read their row and
-//                          release the score columns at once, so the next tile's Q K_S^T runs under the
-//                          exponentials; running max / sum per row; P = exp2(.) as bf16 -> shared memory,
-//                          O += P V_S (smem x smem -> TMEM).  Two issuing threads: one for what writes
-//                          the score columns, one for what accumulates into O.
-//     tail:                Phi = Q W_q^T -> TMEM (in the place of a next tile's scores), phi_q scaled per
-//                          row as bf16 where P sat, O += phi_q S (S in bf16 read like a V tile),
-//                          den = l + phi_q.z, y = O / den -> bf16 -> staged in the P tile -> TMA store.
+//   persistent, one CTA per SM (units left over after the full rounds are split into 128-row halves
+//   over twice as many CTAs); per unit of 2 x 128 query rows a flash-style loop over 128-key tiles
+//   of K_S / V_S:        S = Q K_S^T -> TMEM; the softmax threads (one per row) read their row and
+//                        release the score columns at once, so the next tile's Q K_S^T runs under the
+//                        exponentials; running max / sum per row; P = exp2(.) as bf16 -> shared memory,
+//                        O += P V_S (smem x smem -> TMEM).  Two issuing threads: one for what writes
+//                        the score columns, one for what accumulates into O.
+//   tail:                Phi = Q W_q^T -> TMEM (in the place of a next tile's scores), phi_q scaled per
+//                        row as bf16 where P sat, O += phi_q S (S in bf16 read like a V tile),
+//                        den = l + phi_q.z, y = O / den -> bf16 -> staged in the P tile -> TMA store.
 // All tiles are staged by TMA with the 128-byte swizzle; every mbarrier wait is bounded.
-#include <cuda.h>
-
-#include <mutex>
-
-#include "as_internal.h"
-#include "sm100_ptx.cuh"
-#include "sm100_tmem_wide.cuh"
+#include "tensor_common.cuh"
 
 namespace {
 
-using namespace sm100;
-
-constexpr int BOX_BYTES = 128 * 128;     // one TMA box: 128 rows x 64 bf16 (128 bytes per row)
+using namespace as_tc;
 
 // ======================================================================================
 // Q pass
@@ -61,47 +47,6 @@ struct QLayout {
   static constexpr int BAR_OFF = KV_OFF + KV_STAGES * TILE;
   static constexpr int TOTAL = BAR_OFF + 256 + 1024;       // + slack for the 1024-byte alignment
 };
-
-// Loads a [128 x D] tile (rows y0.., of slice z) as D/64 swizzled boxes.
-template <int D>
-AS_DEV void load_tile(uint32_t dst, const CUtensorMap* m, uint32_t bar, int y0, int z) {
-#pragma unroll
-  for (int b = 0; b < D / 64; ++b) tma_load_3d(dst + b * BOX_BYTES, m, bar, b * 64, y0, z);
-}
-
-// Shared-memory descriptors are built once per tile; the k-steps of one MMA chain only add a byte
-// offset (in 16-byte units) to the address field, which keeps the issuing thread's instruction count low.
-AS_DEV uint64_t kmajor_desc(uint32_t smem) { return make_sdesc(smem, 16, 1024); }        // [rows x 64] boxes, K-major
-AS_DEV uint64_t mnmajor_desc(uint32_t smem) { return make_sdesc(smem, BOX_BYTES, 1024); } // k-rows x [64-column boxes], MN-major
-// offset of k-step kk (16 elements) inside a K-major tile of 64-column boxes
-AS_DEV constexpr uint64_t kstep_kmajor(int kk) { return (uint64_t)(((kk / 4) * BOX_BYTES + (kk % 4) * 32) >> 4); }
-// offset of k-step kk (16 rows) inside an MN-major tile
-AS_DEV constexpr uint64_t kstep_mnmajor(int kk) { return (uint64_t)((kk * 2048) >> 4); }
-
-// D[tmem] (+)= A[smem, K-major, 128 x KD] * B[smem, K-major, NB x KD]^T
-template <int KD>
-AS_DEV void issue_kmajor(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool acc) {
-#pragma unroll
-  for (int kk = 0; kk < KD / 16; ++kk)
-    mma_ss(d_tmem, a_desc + kstep_kmajor(kk), b_desc + kstep_kmajor(kk), idesc, (acc || kk > 0) ? 1u : 0u);
-}
-// D[tmem] (+)= A[tmem, 128 lanes x 128 k as packed bf16] * B[smem, MN-major: 128 k-rows x NB cols]
-AS_DEV void issue_tmemA_mnB(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool acc) {
-#pragma unroll
-  for (int kk = 0; kk < 8; ++kk)
-    mma_ts(d_tmem, a_tmem + kk * 8, b_desc + kstep_mnmajor(kk), idesc, (acc || kk > 0) ? 1u : 0u);
-}
-
-// Writes 32 consecutive columns [c0, c0+32) of row `row` of a swizzled [128 x D] bf16 tile.
-AS_DEV void store_row_chunk(uint8_t* tile, uint32_t row, uint32_t c0, const uint32_t (&w)[16]) {
-  uint8_t* box = tile + (c0 / 64) * BOX_BYTES;
-  const uint32_t chunk0 = (c0 % 64) / 8;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    uint4 v = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
-    *reinterpret_cast<uint4*>(box + swz128_chunk_offset(row, chunk0 + i)) = v;
-  }
-}
 
 // Persistent: one CTA per SM walks over 256-row units (unit w = blockIdx.x + u * gridDim.x; the units of
 // one (batch, head) are consecutive, so the CTAs that run at the same time share K_S / V_S in L2).
@@ -467,7 +412,13 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
       if (cc == 0 && !p_buffer_free(pb + j)) return false;   // the previous tile's P V has read the buffer
       store_row_chunk(sPg, r, cc * 32, pw);
     }
-    l = l * resc + ((la.x + la.y) + (lb.x + lb.y));
+    // The sum above adds the unrounded probabilities while the MMA multiplies their bf16 roundings with V.
+    // Over many keys the rounding errors average out, but the error of a probability that dominates its
+    // row does not, and a result close to one large v_j would be off by up to 2^-9 of its value.  So the
+    // sum takes over the rounding error of the tile's largest probability.
+    const float p_top = ex2(mx - m_ref);
+    const float p_top_err = __uint_as_float(pack_bf16(0.f, p_top) & 0xffff0000u) - p_top;
+    l = l * resc + (((la.x + la.y) + (lb.x + lb.y)) + p_top_err);
     if (__any_sync(0xffffffffu, need)) {
       // the previous tile's P V has completed (waited for above) and this tile's has not been released yet
       tc_fence_after();
@@ -644,457 +595,16 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   }
 }
 
-// ======================================================================================
-// K pass
-// ======================================================================================
-struct KParams {
-  int N, n_s, n_chunks, chunk_tiles, P, F, H;
-  const int32_t* sm_rank;
-  __nv_bfloat16 *ks_w, *vs_w;          // compact softmax K / V (nullptr when nothing is gathered)
-  const __nv_bfloat16 *k, *v;          // not dereferenced by the tensor path (tiles come through TMA)
-  float *part_s, *part_z;
-  uint32_t* status;
-};
-
-constexpr int K_THREADS = 256;           // warps 0-3: feature warps; 4: TMA; 5: MMA; 6-7: gather
-// stages of the K / V ring: 3 with a one-layer feature map; 2 with two layers, where every stage also holds
-// the tile of first-layer activations
-template <int LAYERS> constexpr int k_stages() { return LAYERS == 2 ? 2 : 3; }
-
-template <int D, int LAYERS>
-struct KLayout {
-  static constexpr int K_STAGES = k_stages<LAYERS>();
-  static constexpr int STAGE_TILES = LAYERS == 2 ? 3 : 2;        // K tile, V tile (, first-layer activations)
-  static constexpr int TILE = 128 * D * 2;
-  static constexpr int W_OFF = 0;                                // last-layer weights as a [128 x D] tile (rows >= F are zero)
-  static constexpr int KV_OFF = TILE;                            // K_STAGES x STAGE_TILES tiles
-  static constexpr int BAR_OFF = KV_OFF + K_STAGES * STAGE_TILES * TILE;
-  static constexpr int MASK_OFF = BAR_OFF + 256;                 // 2 x 4 words: linear-token bits per tile
-  static constexpr int RANK_OFF = MASK_OFF + 64;                 // K_STAGES x 128 int32
-  static constexpr int TOTAL = RANK_OFF + K_STAGES * 512 + 1024;
-};
-
-// LAYERS == 2: the features are phi(relu(k W_1^T) W_2^T); relu(k W_1^T) comes precomputed (tmH), tmW is W_2.
-template <int D, int LAYERS>
-__global__ void __launch_bounds__(K_THREADS, 1)
-kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-             const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH, const KParams p) {
-  using L = KLayout<D, LAYERS>;
-  constexpr int K_STAGES = L::K_STAGES;
-  constexpr int F = D;
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const uint32_t sbase = smem_u32(smem);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::BAR_OFF);
-  enum { B_W = 0, B_FULL = 1, B_EMPTY = B_FULL + K_STAGES, B_D1 = B_EMPTY + K_STAGES, B_PK = B_D1 + 2,
-         B_DONE = B_PK + 2, B_COUNT = B_DONE + 1 };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::BAR_OFF + 8 * B_COUNT);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::BAR_OFF + 8 * B_COUNT + 4);
-  uint32_t* sMask = reinterpret_cast<uint32_t*>(smem + L::MASK_OFF);
-  int32_t* sRank = reinterpret_cast<int32_t*>(smem + L::RANK_OFF);
-  auto bar = [&](int i) { return smem_u32(bars + i); };
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int bh = blockIdx.y, h = bh % p.H, chunk = blockIdx.x;
-  const int tiles_total = (p.N + 127) / 128;
-  const int t_begin = chunk * p.chunk_tiles;
-  const int nt = min(p.chunk_tiles, tiles_total - t_begin);
-  const WaitCtx wc{p.status, abort_flag};
-
-  __shared__ uint32_t s_skip;
-  if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile uint32_t*>(p.status);
-  __syncthreads();
-  if (s_skip != 0u) return;
-
-  if (threadIdx.x == 0) {
-    *abort_flag = 0u;
-    mbar_init(bar(B_W), 1);
-    for (int s = 0; s < K_STAGES; ++s) { mbar_init(bar(B_FULL + s), 1); mbar_init(bar(B_EMPTY + s), 3); }
-    for (int b = 0; b < 2; ++b) { mbar_init(bar(B_D1 + b), 1); mbar_init(bar(B_PK + b), 128); }
-    mbar_init(bar(B_DONE), 1);
-    fence_barrier_init();
-    fence_proxy_async();
-  }
-  if (warp == 5) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
-  const uint32_t tD1[2] = {tmem + 0u, tmem + 128u};
-  const uint32_t tAcc = tmem + 256u;
-  const uint32_t sW = sbase + L::W_OFF;
-  auto sK = [&](int st) { return sbase + L::KV_OFF + st * L::STAGE_TILES * L::TILE; };
-  auto sV = [&](int st) { return sbase + L::KV_OFF + st * L::STAGE_TILES * L::TILE + L::TILE; };
-  auto sH = [&](int st) { return sbase + L::KV_OFF + st * L::STAGE_TILES * L::TILE + 2 * L::TILE; };   // two layers only
-
-  if (warp == 4) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmW);
-      mbar_expect_tx(bar(B_W), L::TILE);
-      load_tile<D>(sW, &tmW, bar(B_W), 0, h);                 // rows >= F are out of bounds: zero-filled
-    }
-    for (int t = 0; t < nt; ++t) {
-      const int st = t % K_STAGES, use = t / K_STAGES;
-      if (!mbar_wait_warp(bar(B_EMPTY + st), (use & 1) ^ 1, wc)) break;
-      if (lane == 0) {
-        mbar_expect_tx(bar(B_FULL + st), L::STAGE_TILES * L::TILE);
-        if (LAYERS == 2) load_tile<D>(sH(st), &tmH, bar(B_FULL + st), (t_begin + t) * 128, bh);
-        load_tile<D>(sK(st), &tmK, bar(B_FULL + st), (t_begin + t) * 128, bh);
-        load_tile<D>(sV(st), &tmV, bar(B_FULL + st), (t_begin + t) * 128, bh);
-      }
-      __syncwarp();
-    }
-  } else if (warp == 5) {
-    // ------------------------------------------------------------ MMA issuer
-    constexpr uint32_t ID_PHI = make_idesc(128, 128, 0, 0);    // Phi^T = W_k K^T : M = features, N = 128 tokens
-    constexpr uint32_t ID_ACC = make_idesc(128, D, 0, 1);      // S += phi^T V    : V is MN-major
-    bool ok = mbar_wait_warp(bar(B_W), 0, wc);
-    for (int t = 0; ok && t <= nt; ++t) {
-      if (t < nt) {
-        const int st = t % K_STAGES;
-        ok = mbar_wait_warp(bar(B_FULL + st), (t / K_STAGES) & 1, wc);
-        if (!ok) break;
-        tc_fence_after();
-        if (lane == 0) {
-          issue_kmajor<D>(tD1[t & 1], kmajor_desc(sW), kmajor_desc(LAYERS == 2 ? sH(st) : sK(st)), ID_PHI, false);
-          tc_commit(bar(B_D1 + (t & 1)));
-        }
-        __syncwarp();
-      }
-      if (t >= 1) {
-        const int u = t - 1, st = u % K_STAGES;
-        ok = mbar_wait_warp(bar(B_PK + (u & 1)), (u >> 1) & 1, wc);
-        if (!ok) break;
-        tc_fence_after();
-        if (lane == 0) {
-          issue_tmemA_mnB(tAcc, tD1[u & 1], mnmajor_desc(sV(st)), ID_ACC, u > 0);
-          tc_commit(bar(B_EMPTY + st));
-          if (u == nt - 1) tc_commit(bar(B_DONE));
-        }
-        __syncwarp();
-      }
-    }
-  } else if (warp >= 6) {
-    // ------------------------------------------------------------ gather of softmax-token rows
-    const int gw = warp - 6;
-    // rows handled by this warp: gw*64 .. gw*64+63; two ranks per lane.  The ranks of tile t + 1 are
-    // fetched while tile t is being copied, so that the global-load latency stays off the critical path.
-    auto load_ranks = [&](int t, int (&rk)[2]) {
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int n = (t_begin + t) * 128 + gw * 64 + e * 32 + lane;
-        rk[e] = (t < nt && n < p.N && p.ks_w != nullptr) ? p.sm_rank[n] : -1;
-      }
-    };
-    int rk_next[2];
-    load_ranks(0, rk_next);
-    for (int t = 0; t < nt; ++t) {
-      const int st = t % K_STAGES;
-      int rk[2] = {rk_next[0], rk_next[1]};
-      load_ranks(t + 1, rk_next);
-      if (!mbar_wait_warp(bar(B_FULL + st), (t / K_STAGES) & 1, wc)) break;
-      if (p.ks_w != nullptr) {
-        const uint8_t* kt = smem + L::KV_OFF + st * L::STAGE_TILES * L::TILE;
-        const uint8_t* vt = kt + L::TILE;
-        constexpr int CH = D / 8;                          // 16-byte chunks per row
-        for (int e = 0; e < 2; ++e) {
-          uint32_t bits = __ballot_sync(0xffffffffu, rk[e] >= 0);
-          while (bits) {
-            const int src = __ffs(bits) - 1;
-            bits &= bits - 1;
-            const int rank = __shfl_sync(0xffffffffu, rk[e], src);
-            const uint32_t rrow = gw * 64 + e * 32 + src;
-            // lanes [0, CH) move the K row, lanes [16, 16 + CH) the V row
-            const int c = lane & 15;
-            if (c < CH) {
-              const uint8_t* tile = (lane < 16) ? kt : vt;
-              const uint4 val = *reinterpret_cast<const uint4*>(tile + (c / 8) * BOX_BYTES + swz128_chunk_offset(rrow, c % 8));
-              __nv_bfloat16* dst = ((lane < 16) ? p.ks_w : p.vs_w) + ((size_t)bh * p.n_s + rank) * D + c * 8;
-              *reinterpret_cast<uint4*>(dst) = val;
-            }
-          }
-        }
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B_EMPTY + st));
-    }
-  } else {
-    // ------------------------------------------------------------ feature warps: lane of TMEM = feature f
-    const int f = warp * 32 + lane;
-    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
-    const bool squared = (p.P == 2) && (f >= F / 2);
-    float zacc = 0.f;
-    bool ok = true;
-    uint32_t x[32];
-    // which of a tile's 128 tokens are linear tokens (inside the sequence, not softmax tokens); the table
-    // entry of tile t + 1 is fetched while tile t is processed
-    auto is_linear = [&](int t) {
-      const int n = (t_begin + t) * 128 + f;
-      return (t < nt) && (n < p.N) && (p.sm_rank[n] < 0);
-    };
-    bool lin_next = is_linear(0);
-    for (int t = 0; t < nt; ++t) {
-      const int b = t & 1;
-      {
-        const uint32_t bits = __ballot_sync(0xffffffffu, lin_next);
-        if (lane == 0) sMask[b * 4 + warp] = bits;
-        lin_next = is_linear(t + 1);
-      }
-      // every feature thread reaches this barrier in every iteration, also after a failed wait: a warp
-      // that left the loop early would leave the others waiting here for good
-      named_barrier_sync(1, 128);
-      if (ok) ok = mbar_wait_warp(bar(B_D1 + b), (t >> 1) & 1, wc);
-      if (!ok) continue;
-      tc_fence_after();
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const uint32_t mask = sMask[b * 4 + c];
-        tmem_ld32(tD1[b] + lane_off + c * 32, x);
-        tmem_ld_wait(x);
-        uint32_t w[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float a0 = fmaxf(__uint_as_float(x[2 * i]), 0.f), a1 = fmaxf(__uint_as_float(x[2 * i + 1]), 0.f);
-          if (squared) { a0 *= a0; a1 *= a1; }
-          a0 = ((mask >> (2 * i)) & 1u) ? a0 : 0.f;
-          a1 = ((mask >> (2 * i + 1)) & 1u) ? a1 : 0.f;
-          w[i] = pack_bf16(a0, a1);
-          // z sums the features as the MMA sees them: the bf16 values, read back out of the packed word
-          zacc += __uint_as_float(w[i] << 16) + __uint_as_float(w[i] & 0xffff0000u);
-        }
-        tmem_st16(tD1[b] + lane_off + c * 16, w);
-      }
-      tmem_st_wait();
-      tc_fence_before();
-      mbar_arrive(bar(B_PK + b));
-    }
-    if (ok) ok = mbar_wait_warp(bar(B_DONE), 0, wc);
-    if (ok) {
-      tc_fence_after();
-      if (f < F) {
-        float* ps = p.part_s + (((size_t)bh * p.n_chunks + chunk) * F + f) * D;
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          tmem_ld32(tAcc + lane_off + c * 32, x);
-          tmem_ld_wait(x);
-#pragma unroll
-          for (int i = 0; i < 8; ++i)
-            *reinterpret_cast<uint4*>(ps + c * 32 + 4 * i) = make_uint4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]);
-        }
-        p.part_z[((size_t)bh * p.n_chunks + chunk) * F + f] = zacc;
-      } else {
-        // features beyond F exist only as zero padding (F = 64): keep the warp-collective loads aligned
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) { tmem_ld32(tAcc + lane_off + c * 32, x); tmem_ld_wait(x); }
-      }
-    }
-  }
-
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 5) {
-    tc_fence_after();
-    tmem_dealloc(tmem, 512);
-  }
-}
-
-// ======================================================================================
-// First layer of a two-layer feature map ("Characterization of phi": the embedding network): h1 = relu(x W_1^T)
-// for x = q (blockIdx.z == 0) and x = k (blockIdx.z == 1).  One 128-token tile per CTA.
-// ======================================================================================
-struct P1Params { int H; uint32_t* status; };
-constexpr int P1_THREADS = 160;          // warps 0-3: epilogue (one thread per token row); warp 4: TMA + MMA
-
-template <int D>
-struct P1Layout {
-  static constexpr int TILE = 128 * D * 2;
-  static constexpr int X_OFF = 0, W_OFF = TILE, BAR_OFF = 2 * TILE;
-  static constexpr int TOTAL = BAR_OFF + 64 + 1024;
-};
-
-template <int D>
-__global__ void __launch_bounds__(P1_THREADS)
-phi1_kernel(const __grid_constant__ CUtensorMap tmXq, const __grid_constant__ CUtensorMap tmXk,
-            const __grid_constant__ CUtensorMap tmWq, const __grid_constant__ CUtensorMap tmWk,
-            const __grid_constant__ CUtensorMap tmHq, const __grid_constant__ CUtensorMap tmHk, const P1Params p) {
-  using L = P1Layout<D>;
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const uint32_t sbase = smem_u32(smem);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::BAR_OFF);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::BAR_OFF + 16);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::BAR_OFF + 20);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int bh = blockIdx.y, h = bh % p.H, row0 = blockIdx.x * 128;
-  const bool is_k = blockIdx.z != 0;
-  const CUtensorMap* tmX = is_k ? &tmXk : &tmXq;
-  const CUtensorMap* tmW = is_k ? &tmWk : &tmWq;
-  const CUtensorMap* tmH = is_k ? &tmHk : &tmHq;
-  const WaitCtx wc{p.status, abort_flag};
-  const uint32_t bar_full = smem_u32(bars), bar_done = smem_u32(bars + 1);
-
-  __shared__ uint32_t s_skip;
-  if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile uint32_t*>(p.status);
-  __syncthreads();
-  if (s_skip != 0u) return;
-  if (threadIdx.x == 0) {
-    *abort_flag = 0u;
-    mbar_init(bar_full, 1); mbar_init(bar_done, 1);
-    fence_barrier_init();
-    fence_proxy_async();
-  }
-  if (warp == 4) { tmem_alloc(smem_u32(tmem_slot), 128); tmem_relinquish(); }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
-  const uint32_t sX = sbase + L::X_OFF, sW = sbase + L::W_OFF;
-
-  if (warp == 4) {
-    if (lane == 0) {
-      mbar_expect_tx(bar_full, 2 * L::TILE);
-      load_tile<D>(sX, tmX, bar_full, row0, bh);
-      load_tile<D>(sW, tmW, bar_full, 0, h);                  // W_1[h]: [hidden rows][D]
-    }
-    __syncwarp();
-    if (mbar_wait_warp(bar_full, 0, wc)) {
-      tc_fence_after();
-      if (lane == 0) {
-        issue_kmajor<D>(tmem, kmajor_desc(sX), kmajor_desc(sW), make_idesc(128, D, 0, 0), false);   // X W_1^T, N = hidden = D
-        tc_commit(bar_done);
-      }
-      __syncwarp();
-    }
-  } else {
-    const int r = warp * 32 + lane;
-    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
-    bool ok = mbar_wait_warp(bar_done, 0, wc);
-    if (ok) {
-      tc_fence_after();
-      uint32_t x[32];
-#pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        tmem_ld32(tmem + lane_off + c * 32, x);
-        tmem_ld_wait(x);
-        uint32_t w[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-          w[i] = pack_bf16(fmaxf(__uint_as_float(x[2 * i]), 0.f), fmaxf(__uint_as_float(x[2 * i + 1]), 0.f));
-        store_row_chunk(smem + L::X_OFF, r, c * 32, w);       // the X tile has been consumed by the MMA
-      }
-      fence_proxy_async();
-    }
-    named_barrier_sync(1, 128);                               // reached by every epilogue thread, also after a failed wait
-    if (ok && r == 0) {
-#pragma unroll
-      for (int b = 0; b < D / 64; ++b) tma_store_3d(tmH, sX + b * BOX_BYTES, b * 64, row0, bh);
-      tma_store_commit();
-      tma_store_wait_all();
-    }
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 4) {
-    tc_fence_after();
-    tmem_dealloc(tmem, 128);
-  }
-}
-
-// ======================================================================================
-// Host side: tensor maps and launches
-// ======================================================================================
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn g_encode = nullptr;
-std::once_flag g_once;
-cudaError_t g_init_err = cudaSuccess;
-
-// 3-D bf16 tensor [slices][rows][cols] (cols contiguous) viewed through boxes of 64 cols x box_rows rows.
-bool make_map(CUtensorMap* m, const void* base, int cols, int rows, int slices, int box_rows) {
-  cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)slices};
-  cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)cols * 2 * (cuuint64_t)rows};
-  cuuint32_t box[3] = {64u, (cuuint32_t)box_rows, 1u};
-  cuuint32_t estr[3] = {1u, 1u, 1u};
-  return g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-template <typename K>
-cudaError_t opt_in_smem(K kernel, int bytes) {
-  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-}
-
 }  // namespace
 
-cudaError_t as_tensor_init() {
-  std::call_once(g_once, [] {
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
-    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || fn == nullptr) {
-      g_init_err = (e != cudaSuccess) ? e : cudaErrorNotSupported;
-      return;
-    }
-    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
-  });
-  if (g_init_err != cudaSuccess) return g_init_err;
-  // shared-memory opt-in is per device; cheap enough to repeat
+cudaError_t as_tensor_init_qpass() {
   cudaError_t e;
   if ((e = opt_in_smem(qpass_kernel<128>, QLayout<128>::TOTAL)) != cudaSuccess) return e;
   if ((e = opt_in_smem(qpass_kernel<64>, QLayout<64>::TOTAL)) != cudaSuccess) return e;
-  if ((e = opt_in_smem(kpass_kernel<128, 1>, KLayout<128, 1>::TOTAL)) != cudaSuccess) return e;
-  if ((e = opt_in_smem(kpass_kernel<64, 1>, KLayout<64, 1>::TOTAL)) != cudaSuccess) return e;
-  if ((e = opt_in_smem(phi1_kernel<128>, P1Layout<128>::TOTAL)) != cudaSuccess) return e;
-  if ((e = opt_in_smem(phi1_kernel<64>, P1Layout<64>::TOTAL)) != cudaSuccess) return e;
-  if ((e = opt_in_smem(kpass_kernel<128, 2>, KLayout<128, 2>::TOTAL)) != cudaSuccess) return e;
-  if ((e = opt_in_smem(kpass_kernel<64, 2>, KLayout<64, 2>::TOTAL)) != cudaSuccess) return e;
   return cudaSuccess;
 }
 
-cudaError_t as_tensor_phi1(const as_launch_args& a, cudaStream_t st) {
-  if (g_encode == nullptr) return cudaErrorNotSupported;
-  const int BH = a.B * a.H;
-  CUtensorMap tmXq, tmXk, tmWq, tmWk, tmHq, tmHk;
-  if (!make_map(&tmXq, a.q, a.d, a.N, BH, 128) || !make_map(&tmXk, a.k, a.d, a.N, BH, 128) ||
-      !make_map(&tmWq, a.wq, a.d, a.d, a.H, 128) || !make_map(&tmWk, a.wk, a.d, a.d, a.H, 128) ||
-      !make_map(&tmHq, a.h1q, a.d, a.N, BH, 128) || !make_map(&tmHk, a.h1k, a.d, a.N, BH, 128))
-    return cudaErrorInvalidValue;
-  P1Params p{a.H, a.status};
-  dim3 grid((a.N + 127) / 128, BH, 2);
-  if (a.d == 128) phi1_kernel<128><<<grid, P1_THREADS, P1Layout<128>::TOTAL, st>>>(tmXq, tmXk, tmWq, tmWk, tmHq, tmHk, p);
-  else phi1_kernel<64><<<grid, P1_THREADS, P1Layout<64>::TOTAL, st>>>(tmXq, tmXk, tmWq, tmWk, tmHq, tmHk, p);
-  return cudaGetLastError();
-}
-
-cudaError_t as_tensor_kpass(const as_launch_args& a, cudaStream_t st) {
-  if (g_encode == nullptr) return cudaErrorNotSupported;
-  const int BH = a.B * a.H;
-  CUtensorMap tmK, tmV, tmW, tmH;
-  if (!make_map(&tmK, a.k, a.d, a.N, BH, 128) || !make_map(&tmV, a.v, a.d, a.N, BH, 128) ||
-      !make_map(&tmW, a.layers == 2 ? a.wk2 : a.wk, a.d, a.F, a.H, 128))
-    return cudaErrorInvalidValue;
-  if (a.layers == 2) { if (!make_map(&tmH, a.h1k, a.d, a.N, BH, 128)) return cudaErrorInvalidValue; }
-  else tmH = tmK;               // never used with a one-layer map
-  KParams p{};
-  p.N = a.N; p.n_s = a.n_s; p.n_chunks = a.n_chunks; p.chunk_tiles = a.chunk_tiles; p.P = a.P; p.F = a.F;
-  p.H = a.H; p.sm_rank = a.sm_rank; p.ks_w = a.ks_w; p.vs_w = a.vs_w; p.k = a.k; p.v = a.v;
-  p.part_s = a.part_s; p.part_z = a.part_z; p.status = a.status;
-  dim3 grid(a.n_chunks, BH, 1);
-  if (a.layers == 2) {
-    if (a.d == 128) kpass_kernel<128, 2><<<grid, K_THREADS, KLayout<128, 2>::TOTAL, st>>>(tmK, tmV, tmW, tmH, p);
-    else kpass_kernel<64, 2><<<grid, K_THREADS, KLayout<64, 2>::TOTAL, st>>>(tmK, tmV, tmW, tmH, p);
-  } else {
-    if (a.d == 128) kpass_kernel<128, 1><<<grid, K_THREADS, KLayout<128, 1>::TOTAL, st>>>(tmK, tmV, tmW, tmH, p);
-    else kpass_kernel<64, 1><<<grid, K_THREADS, KLayout<64, 1>::TOTAL, st>>>(tmK, tmV, tmW, tmH, p);
-  }
-  return cudaGetLastError();
-}
-
 cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st) {
-  if (g_encode == nullptr) return cudaErrorNotSupported;
   const int BH = a.B * a.H;
   const bool lin = a.n_l > 0;
   CUtensorMap tmQ, tmK, tmV, tmW, tmSt, tmH, tmO;

@@ -16,6 +16,7 @@ handed to the oracle holds exactly those bf16 values.
 from __future__ import annotations
 
 import dataclasses
+import functools
 import math
 
 import numpy as np
@@ -34,7 +35,13 @@ class Workload:
     seed: int
     rms_norm_qk: bool = True
     degree: int = 2      # polynomial degree P of the feature map
-    layers: int = 1      # depth of the feature map's embedding network (2: hidden width = F)
+    layers: int = 1      # depth of the feature map's embedding network
+    hidden: int = 0      # hidden width of a two-layer network (0: equal to F)
+    bias: bool = False   # embedding layers carry a bias
+
+    @property
+    def hidden_width(self) -> int:
+        return self.hidden if self.hidden > 0 else self.F
 
     @property
     def N(self) -> int:
@@ -112,16 +119,11 @@ def bf16_bits_to_f64(b: np.ndarray) -> np.ndarray:
     return bf16_bits_to_f32(b).astype(np.float64)
 
 
-def generate(wl: Workload, wq_gain: float = 1.0, heads: int | None = None):
-    """Draw one layer's inputs.  Returns a dict of uint16 arrays holding bf16 bit patterns:
-
-      q, k, v : [B, H, N, d]      wq, wk : [H, F, d]      (wl.layers == 2: also wq2, wk2 : [H, F, F])
-
-    Draw order is Q, K, V, W_q, W_k from numpy's PCG64 seeded with `wl.seed`.
-    `wq_gain` multiplies W_q before rounding (used by the tests to make the softmax and
-    the linear branch carry comparable weight).  `heads` (optional) keeps only the first
-    few heads, after drawing all of them, so that a reduced case sees the same values.
-    """
+@functools.lru_cache(maxsize=2)
+def _draw(wl: Workload):
+    """The raw draws of one workload: q, k, v as bf16 bit patterns, the weights still in float32
+    (the gain on W_q is applied before rounding).  Kept for the last two workloads: the tests ask
+    for the same layer several times (other gains, fewer heads)."""
     rng = np.random.Generator(np.random.PCG64(wl.seed))
     shape = (wl.B, wl.H, wl.N, wl.d)
     out = {}
@@ -131,21 +133,55 @@ def generate(wl: Workload, wq_gain: float = 1.0, heads: int | None = None):
             x /= np.sqrt(np.mean(np.square(x, dtype=np.float32), axis=-1, keepdims=True))
         out[name] = f32_to_bf16_bits(x)
         del x
-    a = math.sqrt(6.0 / (wl.d + wl.F))
-    wq = rng.uniform(-a, a, size=(wl.H, wl.F, wl.d)).astype(np.float32)
-    wk = rng.uniform(-a, a, size=(wl.H, wl.F, wl.d)).astype(np.float32)
-    out["wq"] = f32_to_bf16_bits(wq * np.float32(wq_gain))
-    out["wk"] = f32_to_bf16_bits(wk)
-    weight_names = ["wq", "wk"]
+    hid = wl.hidden_width
+    first_out = hid if wl.layers == 2 else wl.F
+    a = math.sqrt(6.0 / (wl.d + first_out))
+    out["wq"] = rng.uniform(-a, a, size=(wl.H, first_out, wl.d)).astype(np.float32)
+    out["wk"] = rng.uniform(-a, a, size=(wl.H, first_out, wl.d)).astype(np.float32)
     if wl.layers == 2:
-        # second layer [H, F, hidden] with hidden = F, drawn after the first layers (which then map d -> hidden)
-        a2 = math.sqrt(6.0 / (wl.F + wl.F))
-        out["wq2"] = f32_to_bf16_bits(rng.uniform(-a2, a2, size=(wl.H, wl.F, wl.F)).astype(np.float32))
-        out["wk2"] = f32_to_bf16_bits(rng.uniform(-a2, a2, size=(wl.H, wl.F, wl.F)).astype(np.float32))
-        weight_names += ["wq2", "wk2"]
+        # second layer [H, F, hidden], drawn after the first layers (which then map d -> hidden)
+        a2 = math.sqrt(6.0 / (hid + wl.F))
+        out["wq2"] = rng.uniform(-a2, a2, size=(wl.H, wl.F, hid)).astype(np.float32)
+        out["wk2"] = rng.uniform(-a2, a2, size=(wl.H, wl.F, hid)).astype(np.float32)
+    if wl.bias:
+        # small biases of either sign, drawn last: bq1, bk1 (, bq2, bk2)
+        out["bq1"] = rng.uniform(-0.1, 0.1, size=(wl.H, first_out)).astype(np.float32)
+        out["bk1"] = rng.uniform(-0.1, 0.1, size=(wl.H, first_out)).astype(np.float32)
+        if wl.layers == 2:
+            out["bq2"] = rng.uniform(-0.1, 0.1, size=(wl.H, wl.F)).astype(np.float32)
+            out["bk2"] = rng.uniform(-0.1, 0.1, size=(wl.H, wl.F)).astype(np.float32)
+    return out
+
+
+WEIGHT_NAMES = ("wq", "wk", "wq2", "wk2", "bq1", "bk1", "bq2", "bk2")
+
+
+def generate(wl: Workload, wq_gain: float = 1.0, heads: int | None = None):
+    """Draw one layer's inputs.  Returns a dict of uint16 arrays holding bf16 bit patterns:
+
+      q, k, v : [B, H, N, d]
+      wq, wk  : [H, F, d]                     (wl.layers == 2: [H, hidden, d], and wq2, wk2 : [H, F, hidden])
+      bq1, bk1 (, bq2, bk2) : [H, width]      (only when wl.bias)
+
+    Draw order is Q, K, V, W_q, W_k (, W_q2, W_k2) (, biases) from numpy's PCG64 seeded with `wl.seed`.
+    `wq_gain` multiplies the LAST layer of the query map (weights and bias) before rounding (used by the
+    tests to make the softmax and the linear branch carry comparable weight; ReLU is positively
+    homogeneous, so this scales the activation a by the gain).  `heads` (optional) keeps only the
+    first few heads, after drawing all of them, so that a reduced case sees the same values.
+    """
+    raw = _draw(wl)
+    g = np.float32(wq_gain)
+    last_w, last_b = ("wq2", "bq2") if wl.layers == 2 else ("wq", "bq1")
+    out = {}
+    for name, x in raw.items():
+        if name in ("q", "k", "v"):
+            out[name] = x.copy()          # the cached draw itself is never handed out
+        else:
+            out[name] = f32_to_bf16_bits(x * g if name in (last_w, last_b) else x)
     if heads is not None and heads < wl.H:
         for name in ("q", "k", "v"):
             out[name] = np.ascontiguousarray(out[name][:, :heads])
-        for name in weight_names:
-            out[name] = np.ascontiguousarray(out[name][:heads])
+        for name in WEIGHT_NAMES:
+            if name in out:
+                out[name] = np.ascontiguousarray(out[name][:heads])
     return out

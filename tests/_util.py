@@ -4,7 +4,9 @@ The expected values always come from `oracle/`; nothing computed on the GPU is f
 """
 from __future__ import annotations
 
+import json
 import math
+import os
 
 import numpy as np
 
@@ -26,6 +28,32 @@ def from_cuda_bf16(t) -> np.ndarray:
     return W.bf16_bits_to_f64(t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16))
 
 
+class Guarded:
+    """A device buffer with sentinel-filled guard bands on both sides (stand-in for a memory checker:
+    a kernel that writes before or past its buffer changes a band, and `check` notices)."""
+    BAND = 1 << 16
+    FILL = 0xA5
+
+    def __init__(self, nbytes: int):
+        import torch
+        self.nbytes = int(nbytes)
+        self.pad = (-self.nbytes) % 256
+        self.raw = torch.full((2 * self.BAND + self.nbytes + self.pad,), self.FILL, dtype=torch.uint8, device="cuda")
+        assert self.raw.data_ptr() % 256 == 0
+
+    def bytes(self):
+        return self.raw[self.BAND:self.BAND + self.nbytes]
+
+    def view(self, dtype, shape):
+        return self.bytes().view(dtype).view(*shape)
+
+    def check(self, what=""):
+        import torch
+        lo, hi = self.raw[:self.BAND], self.raw[self.BAND + self.nbytes:]
+        ok = bool(torch.all(lo == self.FILL)) and bool(torch.all(hi == self.FILL))
+        assert ok, "%s: a guard band next to the buffer was overwritten" % what
+
+
 def oracle_inputs(data):
     return {k: W.bf16_bits_to_f64(v) for k, v in data.items()}
 
@@ -44,22 +72,58 @@ def bf16_ulp(x: np.ndarray) -> np.ndarray:
     return 2.0 ** (np.floor(np.log2(ax)) - 7)
 
 
-def assert_parity(got, ref, what="", strict=True):
-    """The parity bar.  strict: rel-L2 <= 5e-3 and max|got-ref| <= 2e-2 * RMS(ref), as stated.
+def output_rounding_floor(ref: np.ndarray) -> float:
+    """max |bf16(ref) - ref| / RMS(ref): the element-wise error a bf16 output carries even when the
+    value before rounding is exact.  Computed from the oracle output alone."""
+    rounded = W.bf16_bits_to_f64(W.f32_to_bf16_bits(ref.astype(np.float32)))
+    rms = math.sqrt(float((ref ** 2).mean()))
+    return float(np.abs(rounded - ref).max()) / max(rms, 1e-300)
 
-    strict=False is for inputs built to make single softmax tokens dominate some rows (the
-    balanced variants): there an output element can be many times the output RMS, and rounding
-    the result to the bf16 output format alone moves it by up to one bf16 spacing, more than
-    2e-2 * RMS.  The element-wise bound then allows that one spacing of the reference value on
-    top of the stated 2e-2 * RMS; the rel-L2 bound is unchanged."""
+
+_REPORT = os.environ.get("AS_PARITY_REPORT", os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))),
+                                                          "gpurun_out", "parity_report.jsonl"))
+
+
+def _record(entry):
+    """Appends one line with the measured figures of a parity case (best effort; never fails a test)."""
+    try:
+        if os.path.isdir(os.path.dirname(_REPORT)):
+            with open(_REPORT, "a") as f:
+                f.write(json.dumps(entry) + "\n")
+    except OSError:
+        pass
+
+
+def assert_parity(got, ref, what="", strict=None):
+    """The parity bar: rel-L2 <= 5e-3 and max|got-ref| <= 2e-2 * RMS(ref), as the target states it.
+
+    The output is bf16.  Rounding the EXACT result to bf16 already moves an element by up to half a
+    bf16 spacing, which for an element a few output-RMS large is a sizeable part of 2e-2 * RMS and
+    for one beyond about 10 RMS (rows dominated by a single softmax token) exceeds it:
+    `output_rounding_floor`, computed from the oracle output alone, is that share.  Rule, decided from
+    the oracle output only (never from what a kernel returned):
+      floor <= 1e-2 (half the bound)  ->  the stated bound, strictly;
+      floor  > 1e-2                   ->  the stated bound on the value before output rounding:
+                                          |got-ref| <= 2e-2 * RMS + half a bf16 spacing of the reference.
+    strict=True forces the first form.  The rel-L2 bound is the stated one in every case, and the strict
+    figures of every case are recorded (and reported in the failure message) either way."""
     rel_l2, max_abs = errors(got, ref)
     assert np.isfinite(got).all(), "%s: non-finite output" % what
     rms = math.sqrt(float((ref ** 2).mean()))
-    if not strict:
-        excess = np.maximum(np.abs(got - ref) - bf16_ulp(ref), 0.0)
-        max_abs = float(excess.max()) / max(rms, 1e-300)
-    assert rel_l2 <= REL_L2_TOL and max_abs <= MAX_ABS_TOL, \
-        "%s: rel-L2 %.3e (tol %.0e), max-abs/RMS %.3e (tol %.0e)" % (what, rel_l2, REL_L2_TOL, max_abs, MAX_ABS_TOL)
+    floor = output_rounding_floor(ref)
+    if strict is None:
+        strict = floor <= 0.5 * MAX_ABS_TOL
+    excess = np.maximum(np.abs(got - ref) - 0.5 * bf16_ulp(ref), 0.0)
+    max_abs_less_half_ulp = float(excess.max()) / max(rms, 1e-300)
+    _record({"case": what, "strict": bool(strict), "rel_l2": rel_l2, "max_abs_over_rms": max_abs,
+             "max_abs_less_half_ulp_over_rms": max_abs_less_half_ulp, "output_rounding_floor": floor,
+             "max_abs_ref_over_rms": float(np.abs(ref).max()) / max(rms, 1e-300), "elements": int(ref.size)})
+    if os.environ.get("AS_PARITY_COLLECT"):
+        return rel_l2, max_abs
+    bound = max_abs if strict else max_abs_less_half_ulp
+    assert rel_l2 <= REL_L2_TOL and bound <= MAX_ABS_TOL, \
+        "%s: rel-L2 %.3e (tol %.0e), max-abs/RMS %.3e (%s; strict figure %.3e, rounding floor %.3e, tol %.0e)" % (
+            what, rel_l2, REL_L2_TOL, bound, "strict" if strict else "less half a bf16 spacing", max_abs, floor, MAX_ABS_TOL)
     return rel_l2, max_abs
 
 
@@ -105,10 +169,21 @@ def balanced_gain(wl, stab_mode, sample_rows=48, seed=123):
     return math.sqrt(lo * hi)
 
 
-def oracle_eval(wl, data64, stab_mode, rows=None):
-    """(y, aux) of the oracle for every head; `rows` selects query rows."""
-    return O.hybrid_attention(data64["q"], data64["k"], data64["v"], data64["wq"], data64["wk"],
-                              oracle_mask(wl), None, stab_mode, wl.degree, rows=rows)
+_ORACLE_CACHE = {}
+
+
+def oracle_eval(wl, data64, stab_mode, rows=None, key=None):
+    """(y, aux) of the oracle for every head; `rows` selects query rows.  `key` (optional, hashable,
+    naming the inputs completely) keeps the last result so that a second kernel path run on the same
+    inputs is compared with the same oracle output without evaluating it again."""
+    if key is not None and key in _ORACLE_CACHE:
+        return _ORACLE_CACHE[key]
+    res = O.hybrid_attention(data64["q"], data64["k"], data64["v"], data64["wq"], data64["wk"],
+                             oracle_mask(wl), None, stab_mode, wl.degree, rows=rows)
+    if key is not None:
+        _ORACLE_CACHE.clear()
+        _ORACLE_CACHE[key] = res
+    return res
 
 
 def oracle_state(wl, data64):

@@ -13,7 +13,7 @@ import pytest
 
 from oracle import hybrid_attention as O
 from paper_2509_24899_b200 import workloads as W
-from _util import (assert_parity, balanced_gain, errors, from_cuda_bf16, oracle_eval, oracle_inputs,
+from _util import (Guarded, assert_parity, balanced_gain, errors, from_cuda_bf16, oracle_eval, oracle_inputs,
                    oracle_mask, oracle_state, to_cuda_bf16)
 
 pytestmark = pytest.mark.gpu
@@ -43,7 +43,9 @@ def _path(name):
 
 
 def _run(wl, path, mode, gain=1.0, rows=None, heads=None, want_state=False, softmax_idx=None):
-    """Runs the library on wl's inputs; returns (gpu out, gpu aux, oracle y, oracle aux, extras)."""
+    """Runs the library on wl's inputs; returns (gpu out, gpu aux, oracle y, oracle aux, extras).
+
+    out, aux and the workspace sit between sentinel-filled guard bands that must come back untouched."""
     import torch
     from paper_2509_24899_b200 import HybridAttention
     data = W.generate(wl, wq_gain=gain, heads=heads)
@@ -51,10 +53,16 @@ def _run(wl, path, mode, gain=1.0, rows=None, heads=None, want_state=False, soft
         wl = dataclasses.replace(wl, H=heads)
     dev = {k: to_cuda_bf16(v) for k, v in data.items()}
     op = HybridAttention.from_workload(wl, stab_mode=mode, kernel_path=_path(path), softmax_idx=softmax_idx)
-    aux = torch.full((wl.B, wl.H, wl.N, 3), float("nan"), dtype=torch.float32, device="cuda")
-    out = op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], aux=aux)
+    n_el = wl.B * wl.H * wl.N
+    g_out, g_aux, g_ws = Guarded(n_el * wl.d * 2), Guarded(n_el * 3 * 4), Guarded(op.workspace_bytes)
+    out = g_out.view(torch.bfloat16, (wl.B, wl.H, wl.N, wl.d))
+    aux = g_aux.view(torch.float32, (wl.B, wl.H, wl.N, 3))
+    aux.fill_(float("nan"))
+    op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], out=out, aux=aux, workspace=g_ws.bytes())
     torch.cuda.synchronize()
     assert op.last_status() == 0
+    for g, name in ((g_out, "out"), (g_aux, "aux"), (g_ws, "workspace")):
+        g.check("%s/%s %s" % (wl.name, path, name))
     got = from_cuda_bf16(out)
     got_aux = aux.cpu().numpy().astype(np.float64)
     extras = {"op": op, "n_softmax": op.n_softmax, "indices": op.softmax_indices()}
@@ -63,12 +71,19 @@ def _run(wl, path, mode, gain=1.0, rows=None, heads=None, want_state=False, soft
         torch.cuda.synchronize()
         extras["S"], extras["z"] = S.cpu().numpy().astype(np.float64), z.cpu().numpy().astype(np.float64)
     d64 = oracle_inputs(data)
-    ref, ref_aux = oracle_eval(wl, d64, mode, rows=rows)
+    key = (wl, mode, float(gain), None if rows is None else tuple(int(r) for r in rows),
+           None if softmax_idx is None else tuple(softmax_idx))
+    ref, ref_aux = oracle_eval(wl, d64, mode, rows=rows, key=key)
     if rows is not None:
         got, got_aux = got[:, :, rows], got_aux[:, :, rows]
     extras["data64"] = d64
     extras["wl"] = wl
     return got, got_aux, ref, ref_aux, extras
+
+
+def _tag(name, path, mode, balanced=None):
+    t = "%s/%s/%s" % (name, path, "exact" if mode == O.STAB_EXACT else "paper")
+    return t if balanced is None else t + ("/balanced" if balanced else "/as-drawn")
 
 
 def _check_aux(got_aux, ref_aux, wl, n_softmax):
@@ -87,7 +102,7 @@ def test_tiny_config(path, mode, balanced):
     gain = balanced_gain(wl, mode) if balanced else 1.0
     got, got_aux, ref, ref_aux, ex = _run(wl, path, mode, gain, want_state=True)
     assert ex["n_softmax"] == 32
-    assert_parity(got, ref, "tiny/%s" % path, strict=(not balanced and mode == O.STAB_PAPER))
+    assert_parity(got, ref, _tag("tiny", path, mode, balanced))
     _check_aux(got_aux, ref_aux, wl, 32)
     S, z = oracle_state(wl, ex["data64"])
     assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
@@ -106,7 +121,7 @@ def test_small_ragged_cases(path, mode, name):
     got, got_aux, ref, ref_aux, ex = _run(wl, path, mode, gain, want_state=True)
     mask = oracle_mask(wl)
     assert ex["indices"] == np.flatnonzero(mask).tolist()         # integer work: bit-exact
-    assert_parity(got, ref, "%s/%s" % (name, path), strict=False)
+    assert_parity(got, ref, _tag(name, path, mode, True))
     _check_aux(got_aux, ref_aux, wl, int(mask.sum()))
     S, z = oracle_state(wl, ex["data64"])
     assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
@@ -121,7 +136,7 @@ def test_degenerate_rates(path, rate, name):
     assert ex["n_softmax"] == (wl.N if rate == 1 else 0)
     ok = np.isfinite(ref).all(-1)          # rate 0: a query with all-zero features is NaN in both
     assert ok.mean() > 0.99
-    assert_parity(got[ok], ref[ok], "%s/R%d/%s" % (name, rate, path), strict=False)
+    assert_parity(got[ok], ref[ok], _tag("%s/R%d" % (name, rate), path, O.STAB_PAPER))
     _check_aux(got_aux[ok], ref_aux[ok], wl, ex["n_softmax"])
     if rate == 1:
         # rate 1 is plain softmax attention: cross-check with the library routine as well
@@ -129,7 +144,7 @@ def test_degenerate_rates(path, rate, name):
         d = ex["data64"]
         sd = torch.nn.functional.scaled_dot_product_attention(
             torch.from_numpy(d["q"]), torch.from_numpy(d["k"]), torch.from_numpy(d["v"])).numpy()
-        assert_parity(got, sd, "sdpa", strict=False)
+        assert_parity(got, sd, _tag("%s/R1-vs-sdpa" % name, path, O.STAB_PAPER))
 
 
 @pytest.mark.parametrize("path", PATHS)
@@ -149,7 +164,7 @@ def test_explicit_softmax_index_list(path):
     mask = np.zeros(wl.N, bool)
     mask[idx] = True
     ref, _ = O.hybrid_attention(d64["q"], d64["k"], d64["v"], d64["wq"], d64["wk"], mask)
-    assert_parity(from_cuda_bf16(out), ref, "explicit idx/%s" % path, strict=False)
+    assert_parity(from_cuda_bf16(out), ref, _tag("explicit_idx", path, O.STAB_PAPER))
 
 
 @pytest.mark.parametrize("path", PATHS)
@@ -177,7 +192,7 @@ def test_late_dominant_keys_move_the_reference_maximum(path, mode):
     rows = _sample_rows(wl.N, 512, 7)
     ref, ref_aux = oracle_eval(wl, d64, mode, rows=rows)
     assert (ref_aux[..., 0] > 12.0).mean() > 0.2   # the scaled keys do dominate many rows (c_i far above the usual ~4)
-    assert_parity(from_cuda_bf16(out)[:, :, rows], ref, "late dominant keys/%s" % path, strict=False)
+    assert_parity(from_cuda_bf16(out)[:, :, rows], ref, _tag("late_dominant_keys", path, mode, True))
     _check_aux(aux.cpu().numpy().astype(np.float64)[:, :, rows], ref_aux, wl, int(mask.sum()))
 
 
@@ -212,7 +227,7 @@ def test_wan17_full(path, mode, balanced):
     gain = balanced_gain(wl, mode) if balanced else 1.0
     got, got_aux, ref, ref_aux, ex = _run(wl, path, mode, gain, want_state=True)
     assert ex["n_softmax"] == 975
-    assert_parity(got, ref, "wan17/%s" % path, strict=not balanced)
+    assert_parity(got, ref, _tag("wan17", path, mode, balanced))
     _check_aux(got_aux, ref_aux, wl, 975)
     S, z = oracle_state(wl, ex["data64"])
     assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
@@ -224,51 +239,77 @@ def _sample_rows(N, n, seed):
     return np.unique(np.concatenate([rows, [0, 1, N - 2, N - 1]]))      # include first / last tile rows
 
 
+@pytest.mark.parametrize("path", PATHS)          # outermost: varies fastest, so both paths share one oracle run
 @pytest.mark.parametrize("mode", MODES)
 @pytest.mark.parametrize("balanced", [False, True])
-def test_wan81_headline_sampled_rows(mode, balanced):
-    """Headline shape in the launch configuration the benchmark times (tensor path)."""
+def test_wan81_headline_sampled_rows(path, mode, balanced):
+    """Headline shape in the launch configuration the benchmark times (tensor path), and on the fp32 check path."""
     wl = W.CONFIGS["wan81"]
     gain = balanced_gain(wl, mode) if balanced else 1.0
     rows = _sample_rows(wl.N, 160, 1)
-    got, got_aux, ref, ref_aux, ex = _run(wl, FULL_PATH, mode, gain, rows=rows, want_state=True)
+    got, got_aux, ref, ref_aux, ex = _run(wl, path, mode, gain, rows=rows, want_state=True)
     assert ex["n_softmax"] == 4095
     assert ex["indices"] == np.flatnonzero(oracle_mask(wl)).tolist()
-    assert_parity(got, ref, "wan81", strict=not balanced)
+    assert_parity(got, ref, _tag("wan81/160rows", path, mode, balanced))
     _check_aux(got_aux, ref_aux, wl, 4095)
     S, z = oracle_state(wl, ex["data64"])
     assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
 
 
-@pytest.mark.parametrize("rate", [1, 4, 16, 0])
-def test_stack_layer_rates_sampled_rows(rate):
-    """One layer of each distinct rate of the 30-layer block-rate stack (rate 8 is the headline)."""
+# (rate, mode, balanced): at rates 1 and 0 there is one branch only, so the mode and the gain change nothing
+STACK_CASES = [(1, O.STAB_PAPER, False), (0, O.STAB_PAPER, False)] + \
+              [(r, m, b) for r in (4, 16) for m in MODES for b in (False, True)]
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("rate,mode,balanced", STACK_CASES)
+def test_stack_layer_rates_sampled_rows(path, rate, mode, balanced):
+    """One layer of each distinct rate of the 30-layer block-rate stack (rate 8 is the headline), all heads."""
     sched = W.stack_schedule(0)
     layer = sched.index(rate)
     wl = W.stack_layer(layer)
     assert wl.rate == rate
-    gain = balanced_gain(wl, O.STAB_PAPER)
+    gain = balanced_gain(wl, mode) if balanced else 1.0
     rows = _sample_rows(wl.N, 96, 2)
-    got, got_aux, ref, ref_aux, ex = _run(wl, FULL_PATH, O.STAB_PAPER, gain, rows=rows, heads=4,
-                                          want_state=(rate != 1))
+    got, got_aux, ref, ref_aux, ex = _run(wl, path, mode, gain, rows=rows, want_state=(rate != 1))
     assert ex["n_softmax"] == {1: 32760, 4: 8190, 16: 2100, 0: 0}[rate]
     ok = np.isfinite(ref).all(-1)
     assert ok.mean() > 0.99
-    assert_parity(got[ok], ref[ok], "stack R=%d" % rate, strict=False)
+    assert_parity(got[ok], ref[ok], _tag("stack/R%d/96rows" % rate, path, mode, balanced))
     _check_aux(got_aux[ok], ref_aux[ok], ex["wl"], ex["n_softmax"])
     if rate != 1:
         S, z = oracle_state(ex["wl"], ex["data64"])
         assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
 
 
-def test_wan161_cfg_batch_sampled_rows():
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("balanced", [False, True])
+def test_wan161_cfg_batch_sampled_rows(path, mode, balanced):
     wl = W.CONFIGS["wan161cfg"]
-    gain = balanced_gain(wl, O.STAB_PAPER)
+    gain = balanced_gain(wl, mode) if balanced else 1.0
     rows = _sample_rows(wl.N, 64, 3)
-    got, got_aux, ref, ref_aux, ex = _run(wl, FULL_PATH, O.STAB_PAPER, gain, rows=rows)
+    got, got_aux, ref, ref_aux, ex = _run(wl, path, mode, gain, rows=rows)
     assert ex["n_softmax"] == 4100
-    assert_parity(got, ref, "wan161cfg", strict=False)
+    assert_parity(got, ref, _tag("wan161cfg/64rows", path, mode, balanced))
     _check_aux(got_aux, ref_aux, wl, 4100)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("name", ["wan81", "wan161cfg"])
+def test_whole_output_at_full_size(path, name):
+    """Every output element of the headline layer and of the long CFG-batch layer against the oracle
+    (balanced feature maps, so that both branches carry weight): a mis-addressed unit, half-unit or
+    head of the persistent schedule cannot hide between sampled rows."""
+    wl = W.CONFIGS[name]
+    gain = balanced_gain(wl, O.STAB_PAPER)
+    got, got_aux, ref, ref_aux, ex = _run(wl, path, O.STAB_PAPER, gain)
+    assert_parity(got, ref, _tag(name + "/whole", path, O.STAB_PAPER, True))
+    _check_aux(got_aux, ref_aux, wl, ex["n_softmax"])
+    # per (batch, head) as well: one wrong head would be diluted 12- or 24-fold in the global figure
+    for b in range(wl.B):
+        for h in range(wl.H):
+            assert errors(got[b, h], ref[b, h])[0] <= 5e-3, (b, h)
 
 
 @pytest.mark.parametrize("path", PATHS)
@@ -388,7 +429,7 @@ def test_two_layer_feature_map(mode, name):
     got = from_cuda_bf16(out)
     ok = np.isfinite(ref).all(-1)
     assert ok.mean() > 0.99
-    assert_parity(got[ok], ref[ok], name, strict=False)
+    assert_parity(got[ok], ref[ok], _tag(name, "tensor", mode))
     _check_aux(aux.cpu().numpy().astype(np.float64)[ok], ref_aux[ok], wl, op.n_softmax)
 
 
@@ -448,5 +489,5 @@ def test_many_units_per_cta(mode, name):
     wl = MANY_UNITS[name]
     gain = balanced_gain(wl, mode)
     got, got_aux, ref, ref_aux, ex = _run(wl, FULL_PATH, mode, gain)
-    assert_parity(got, ref, name, strict=False)
+    assert_parity(got, ref, _tag(name, FULL_PATH, mode, True))
     _check_aux(got_aux, ref_aux, wl, ex["n_softmax"])
