@@ -64,8 +64,10 @@ enum { AS_STAB_PAPER = 0, AS_STAB_EXACT = 1 };
 /* Activation of the feature map's embedding layers. */
 enum { AS_ACT_RELU = 0 };
 
-/* Kernel path.  AS_PATH_TENSOR: tcgen05/TMEM/TMA kernels (the product path).
- * AS_PATH_SIMT: plain fp32 CUDA-core kernels kept as an on-device cross-check. */
+/* Kernel path.  AS_PATH_TENSOR (0, the default) is the library: tcgen05/TMEM/TMA kernels.
+ * AS_PATH_SIMT is a TEST AID, not a second backend: plain fp32 CUDA-core kernels of the same steps, kept so
+ * that the tests can put an fp32 result beside the tensor-core one on the same inputs.  It is slow, covers
+ * one-layer feature maps with F == d and degree <= 2 without bias only, and nothing selects it on its own. */
 enum { AS_PATH_TENSOR = 0, AS_PATH_SIMT = 1 };
 
 /* Kernel classes reported by the profiling calls. */
@@ -83,23 +85,29 @@ typedef struct {
   const int32_t* softmax_idx;      /* optional HOST pointer to an explicit sorted, unique T_S;
                                       NULL selects the rule above                                   */
   int32_t  n_softmax;              /* length of softmax_idx (ignored when it is NULL)              */
-  int32_t  phi_dim;                /* F: output width of the feature map, in {64, 128}, == P * D'   */
-  int32_t  phi_layers;             /* embedding-network depth: 1, or 2 (tensor path, phi_hidden == d) */
-  int32_t  phi_hidden;             /* hidden width when phi_layers == 2 (unused otherwise)          */
-  int32_t  poly_degree;            /* P: part p (1-based) of the activation is raised to power p;
-                                      1 or 2 is supported                                            */
+  int32_t  phi_dim;                /* F == P * D': output width of the feature map.  One layer: d, or a
+                                      multiple of 128 up to 512.  Two layers: see phi_hidden.          */
+  int32_t  phi_layers;             /* embedding-network depth: 1 or 2                                */
+  int32_t  phi_hidden;             /* hidden width when phi_layers == 2 (unused otherwise).  d = 128:
+                                      hidden and F each 128 or 256 (the paper's default map is
+                                      d -> 2d -> 2d); d = 64: hidden == F == 64                        */
+  int32_t  poly_degree;            /* P in 1..4: part p (1-based) of the activation is raised to the
+                                      power p; F / P must be a multiple of 32                          */
   int32_t  phi_act;                /* AS_ACT_RELU                                                   */
   float    softmax_scale;          /* 0 selects 1/sqrt(d)                                           */
   int32_t  stab_mode;              /* AS_STAB_PAPER | AS_STAB_EXACT                                 */
-  int32_t  kernel_path;            /* AS_PATH_TENSOR | AS_PATH_SIMT                                 */
+  int32_t  kernel_path;            /* AS_PATH_TENSOR; AS_PATH_SIMT only in tests (see above)        */
 } as_hybrid_attn_desc_t;
 
 /* Feature-map weights, DEVICE pointers, bf16, row-major with the output feature as the slow
  * index ("Characterization of phi": an embedding network, then the polynomial parts).
- *   phi_layers == 1:  w*1 is [H, F, d];                        a = ReLU(W_1 x)
- *   phi_layers == 2:  w*1 is [H, hidden, d], w*2 is [H, F, hidden];  a = ReLU(W_2 ReLU(W_1 x))
- * phi(x) = [a_1, a_2^2]: a split into P contiguous parts, part p to the power p.  Biases must be
- * NULL in this build; w*2 must be NULL when phi_layers == 1. */
+ *   phi_layers == 1:  w*1 is [H, F, d], b*1 [H, F];                  a = ReLU(W_1 x + b_1)
+ *   phi_layers == 2:  w*1 is [H, hidden, d], b*1 [H, hidden], w*2 is [H, F, hidden], b*2 [H, F];
+ *                     a = ReLU(W_2 ReLU(W_1 x + b_1) + b_2)
+ * phi(x) = [a_1, a_2^2, ..., a_P^P]: a split into P contiguous parts, part p to the power p.
+ * Weight matrices are 16-byte aligned.  Every bias is optional (NULL = none; the paper does not say
+ * whether the embedding layers carry one) and 4-byte aligned; w*2 and b*2 must be NULL when
+ * phi_layers == 1.  With two layers the hidden activations are rounded to bf16 between the layers. */
 typedef struct {
   const void *wq1, *bq1, *wq2, *bq2;
   const void *wk1, *bk1, *wk2, *bk2;
@@ -107,16 +115,20 @@ typedef struct {
 
 /* Creates a handle for one layer geometry on the CURRENT device: validates the descriptor,
  * builds the token split on the host (section "Hybrid Attention", token rule) and uploads the
- * index tables.  Returns AS_ERR_ARCH when the current device is not sm_100. */
+ * index tables.  Returns AS_ERR_ARCH when the current device is not sm_100.  The handle belongs to
+ * that device: forward, forward_host, linear_state and last_status return AS_ERR_INVALID_ARG when
+ * another device is current. */
 AS_API as_status_t as_hybrid_attn_create(const as_hybrid_attn_desc_t* desc, as_hybrid_attn_t* out);
 
-/* Frees the handle and its device tables.  NULL is a no-op. */
+/* Frees the handle and its device tables.  NULL is a no-op.  (Utility: no counterpart in the paper.) */
 AS_API as_status_t as_hybrid_attn_destroy(as_hybrid_attn_t h);
 
-/* Bytes of scratch `forward` needs (compacted softmax K/V, partial and final linear state). */
+/* Bytes of scratch `forward` needs (compacted softmax K/V, partial and final linear state, the keys' hidden
+ * activations of a two-layer map).  (Utility: no counterpart in the paper.) */
 AS_API as_status_t as_hybrid_attn_workspace_bytes(as_hybrid_attn_t h, size_t* bytes);
 
-/* Bytes of scratch `forward_host` needs: the above plus device staging for q, k, v and out. */
+/* Bytes of scratch `forward_host` needs: the above plus device staging for q, k, v and out.
+ * (Utility: no counterpart in the paper.) */
 AS_API as_status_t as_hybrid_attn_workspace_bytes_host(as_hybrid_attn_t h, size_t* bytes);
 
 /* The hybrid attention forward pass (equation above; hybrid equation of the paper).
@@ -158,17 +170,27 @@ AS_API as_status_t as_hybrid_attn_softmax_tokens(as_hybrid_attn_t h, int32_t* co
 
 /* Synchronises `cuda_stream`, then reads and clears the handle's device status word.
  * AS_OK, AS_ERR_DEVICE_TIMEOUT (a bounded barrier wait in a kernel expired; outputs of that
- * forward are undefined but the context stays usable) or AS_ERR_CUDA. */
+ * forward are undefined but the context stays usable) or AS_ERR_CUDA.  After a time-out the handle is
+ * INERT until this call has read and cleared the word: the kernels of every later forward on the handle
+ * return at once and leave their outputs untouched, while `forward` itself keeps returning AS_OK.
+ * (Utility: no counterpart in the paper.) */
 AS_API as_status_t as_hybrid_attn_last_status(as_hybrid_attn_t h, void* cuda_stream);
 
-/* Profiling aid: after `profile_enable(h, 1)` every kernel launch is bracketed by CUDA events on
+/* Test aid (no counterpart in the paper): enqueues a one-CTA kernel that waits, with the same bounded wait
+ * every kernel of the library uses, on a barrier nobody arrives at; no copy and no tensor-core operation is
+ * in flight.  After about `limit_cycles` SM clocks (1 .. 1e8) the wait gives up, the kernel returns and the
+ * handle's status word is set exactly as by a time-out inside `forward`: as_hybrid_attn_last_status then
+ * returns AS_ERR_DEVICE_TIMEOUT once, and the handle is usable again afterwards. */
+AS_API as_status_t as_hybrid_attn_debug_expire_wait(as_hybrid_attn_t h, int64_t limit_cycles, void* cuda_stream);
+
+/* Profiling aid (no counterpart in the paper): after `profile_enable(h, 1)` every kernel launch is bracketed by CUDA events on
  * the launching stream.  `profile_read` synchronises those events, adds the elapsed device time
  * per kernel class into ms[AS_NUM_KERNELS] and the launch counts into launches[AS_NUM_KERNELS],
  * and resets the counters.  At most 1024 launches are kept between two reads. */
 AS_API as_status_t as_hybrid_attn_profile_enable(as_hybrid_attn_t h, int32_t enable);
 AS_API as_status_t as_hybrid_attn_profile_read(as_hybrid_attn_t h, float* ms, int32_t* launches);
 
-/* Total number of kernels this handle has launched since create. */
+/* Total number of kernels this handle has launched since create.  (Utility: no counterpart in the paper.) */
 AS_API as_status_t as_hybrid_attn_launch_count(as_hybrid_attn_t h, uint64_t* count);
 
 /* The linear state S, z of one layer, computed WITHOUT allocating anything.  The paper has no
@@ -177,7 +199,12 @@ AS_API as_status_t as_hybrid_attn_launch_count(as_hybrid_attn_t h, uint64_t* cou
  * may only touch the buffers its host framework handed it, a latency-critical loop that must
  * avoid the device-wide synchronisation inside cudaMalloc / cudaFree.  It needs no handle and
  * no workspace: the per-chunk partial sums live in a fixed 8 MiB array inside the library
- * image (every GPU that loads the library holds it until the process exits).
+ * image.  The CUDA driver sets that array up on a device when the library's code is first loaded
+ * there - with the default lazy module loading that is this function's first call on the device,
+ * with CUDA_MODULE_LOADING=EAGER it is context creation - and keeps it until the process exits.
+ * A caller whose arena is about to take all of the device's memory therefore makes one call per
+ * device beforehand (or sets CUDA_MODULE_LOADING=EAGER); if the 8 MiB cannot be had any more, that
+ * first call returns AS_ERR_CUDA and launches nothing.
  *   k, v      [B,H,N,d] bf16 device, read only          wk  [H,d,d] bf16 device (F == d, one layer)
  *   grid_*, blk_*, rate_den, poly_degree                 as in as_hybrid_attn_desc_t (rule-based T_S)
  *   S_out     [B,H,d,d] fp32 device, written             z_out [B,H,d] fp32 device, written
@@ -215,7 +242,7 @@ AS_API as_status_t as_select_block_rates(int32_t n_blocks, int32_t n_rates, cons
                                          double budget, int32_t* choice_out, double* total_cost_out,
                                          double* total_err_out);
 
-/* Static description of a status code. */
+/* Static description of a status code.  (Utility: no counterpart in the paper.) */
 AS_API const char* as_status_string(as_status_t s);
 
 #ifdef __cplusplus

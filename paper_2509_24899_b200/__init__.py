@@ -17,11 +17,12 @@ class HybridAttention:
     """One layer geometry bound to the current CUDA device.
 
     q, k, v: torch.bfloat16 CUDA tensors [B, H, N, d]; wq, wk: bfloat16 [H, F, d]; with phi_layers=2 the
-    feature map is relu(relu(x wq^T) wq2^T) before the powers, wq2, wk2: bfloat16 [H, F, F].
+    feature map is relu(relu(x wq^T + bq1) wq2^T + bq2) before the powers, wq, wk: [H, hidden, d], wq2, wk2:
+    bfloat16 [H, F, hidden].  Biases (optional, bfloat16 [H, width]) are passed as `biases={"bq1": t, ...}`.
     """
 
     def __init__(self, B, H, N, d, grid, block, rate, phi_dim=None, poly_degree=2, softmax_scale=0.0,
-                 stab_mode=AS_STAB_PAPER, kernel_path=AS_PATH_TENSOR, softmax_idx=None, phi_layers=1):
+                 stab_mode=AS_STAB_PAPER, kernel_path=AS_PATH_TENSOR, softmax_idx=None, phi_layers=1, phi_hidden=None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("HybridAttention needs a CUDA device; there is no CPU fallback")
@@ -30,7 +31,7 @@ class HybridAttention:
         self.rate = rate
         self._desc = binding.make_desc(B, H, N, d, grid, block, rate, phi_dim, poly_degree, softmax_scale,
                                        stab_mode, kernel_path, softmax_idx, phi_layers=phi_layers,
-                                       phi_hidden=self.F if phi_layers == 2 else 0)
+                                       phi_hidden=(phi_hidden or self.F) if phi_layers == 2 else 0)
         self._h = binding.as_hybrid_attn_create(self._desc)
         self.workspace_bytes = binding.as_hybrid_attn_workspace_bytes(self._h)
         self.workspace_bytes_host = binding.as_hybrid_attn_workspace_bytes_host(self._h)
@@ -40,7 +41,7 @@ class HybridAttention:
     @classmethod
     def from_workload(cls, wl, **kw):
         return cls(wl.B, wl.H, wl.N, wl.d, wl.grid, wl.block, wl.rate, phi_dim=wl.F,
-                   poly_degree=wl.degree, phi_layers=getattr(wl, "layers", 1), **kw)
+                   poly_degree=wl.degree, phi_layers=wl.layers, phi_hidden=wl.hidden_width, **kw)
 
     @property
     def handle(self):
@@ -57,7 +58,7 @@ class HybridAttention:
         return binding.as_hybrid_attn_softmax_tokens(self._h)[1]
 
     def forward(self, q, k, v, wq=None, wk=None, out=None, aux=None, stream=None, wq2=None, wk2=None,
-                workspace=None):
+                workspace=None, biases=None):
         """`workspace` (optional): a caller-owned uint8 CUDA tensor of at least `workspace_bytes`, 256-byte
         aligned; it becomes the handle's workspace for `linear_state` as well."""
         import torch
@@ -71,18 +72,21 @@ class HybridAttention:
             self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(),
             0 if wq is None else wq.data_ptr(), 0 if wk is None else wk.data_ptr(),
             out.data_ptr(), 0 if aux is None else aux.data_ptr(), ws.data_ptr(), ws.numel(), st.cuda_stream,
-            0 if wq2 is None else wq2.data_ptr(), 0 if wk2 is None else wk2.data_ptr())
+            0 if wq2 is None else wq2.data_ptr(), 0 if wk2 is None else wk2.data_ptr(),
+            None if biases is None else {n: t.data_ptr() for n, t in biases.items()})
         return out
 
-    def forward_host(self, q_host, k_host, v_host, wq, wk, out_host, stream=None):
-        """q_host, k_host, v_host, out_host: pinned CPU tensors; wq, wk: device tensors."""
+    def forward_host(self, q_host, k_host, v_host, wq, wk, out_host, stream=None, wq2=None, wk2=None, biases=None):
+        """q_host, k_host, v_host, out_host: pinned CPU tensors; the weights are device tensors."""
         import torch
         ws = self.workspace(host=True)
         st = torch.cuda.current_stream() if stream is None else stream
         binding.as_hybrid_attn_forward_host(
             self._h, q_host.data_ptr(), k_host.data_ptr(), v_host.data_ptr(),
             0 if wq is None else wq.data_ptr(), 0 if wk is None else wk.data_ptr(),
-            out_host.data_ptr(), ws.data_ptr(), ws.numel(), st.cuda_stream)
+            out_host.data_ptr(), ws.data_ptr(), ws.numel(), st.cuda_stream,
+            0 if wq2 is None else wq2.data_ptr(), 0 if wk2 is None else wk2.data_ptr(),
+            None if biases is None else {n: t.data_ptr() for n, t in biases.items()})
         return out_host
 
     def linear_state(self, stream=None):

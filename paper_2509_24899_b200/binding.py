@@ -71,6 +71,7 @@ def lib() -> C.CDLL:
             "as_hybrid_attn_linear_state": [H, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
             "as_hybrid_attn_softmax_tokens": [H, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.c_int32],
             "as_hybrid_attn_last_status": [H, C.c_void_p],
+            "as_hybrid_attn_debug_expire_wait": [H, C.c_int64, C.c_void_p],
             "as_hybrid_attn_profile_enable": [H, C.c_int32],
             "as_hybrid_attn_profile_read": [H, C.POINTER(C.c_float), C.POINTER(C.c_int32)],
             "as_hybrid_attn_launch_count": [H, C.POINTER(C.c_uint64)],
@@ -143,27 +144,30 @@ def as_hybrid_attn_workspace_bytes_host(h) -> int:
     return n.value
 
 
-def _weights(wq_ptr, wk_ptr, wq2_ptr=0, wk2_ptr=0):
+def _weights(wq_ptr, wk_ptr, wq2_ptr=0, wk2_ptr=0, biases=None):
+    """as_phi_weights_t from integer device addresses; `biases` maps 'bq1', 'bk1', 'bq2', 'bk2' to addresses."""
     if not wq_ptr and not wk_ptr:
         return None
     w = as_phi_weights_t()
     w.wq1, w.wk1 = wq_ptr, wk_ptr
     w.wq2, w.wk2 = wq2_ptr or None, wk2_ptr or None
+    for name, ptr in (biases or {}).items():
+        setattr(w, name, ptr or None)
     return C.byref(w)
 
 
 def as_hybrid_attn_forward(h, q_ptr, k_ptr, v_ptr, wq_ptr, wk_ptr, out_ptr, aux_ptr, ws_ptr, ws_bytes,
-                           stream_ptr, wq2_ptr=0, wk2_ptr=0) -> None:
+                           stream_ptr, wq2_ptr=0, wk2_ptr=0, biases=None) -> None:
     """All pointers are integer device addresses (e.g. tensor.data_ptr()); 0 / None means NULL.
-    wq2_ptr / wk2_ptr: second-layer weights of a two-layer feature map."""
-    _check(lib().as_hybrid_attn_forward(h, q_ptr, k_ptr, v_ptr, _weights(wq_ptr, wk_ptr, wq2_ptr, wk2_ptr), out_ptr, aux_ptr or None,
-                                        ws_ptr, ws_bytes, stream_ptr or None), "as_hybrid_attn_forward")
+    wq2_ptr / wk2_ptr: second-layer weights of a two-layer feature map; biases: dict of addresses."""
+    _check(lib().as_hybrid_attn_forward(h, q_ptr, k_ptr, v_ptr, _weights(wq_ptr, wk_ptr, wq2_ptr, wk2_ptr, biases), out_ptr,
+                                        aux_ptr or None, ws_ptr, ws_bytes, stream_ptr or None), "as_hybrid_attn_forward")
 
 
 def as_hybrid_attn_forward_host(h, q_host, k_host, v_host, wq_ptr, wk_ptr, out_host, ws_ptr, ws_bytes,
-                                stream_ptr, wq2_ptr=0, wk2_ptr=0) -> None:
-    _check(lib().as_hybrid_attn_forward_host(h, q_host, k_host, v_host, _weights(wq_ptr, wk_ptr, wq2_ptr, wk2_ptr), out_host,
-                                             ws_ptr, ws_bytes, stream_ptr or None), "as_hybrid_attn_forward_host")
+                                stream_ptr, wq2_ptr=0, wk2_ptr=0, biases=None) -> None:
+    _check(lib().as_hybrid_attn_forward_host(h, q_host, k_host, v_host, _weights(wq_ptr, wk_ptr, wq2_ptr, wk2_ptr, biases),
+                                             out_host, ws_ptr, ws_bytes, stream_ptr or None), "as_hybrid_attn_forward_host")
 
 
 def as_hybrid_attn_linear_state(h, ws_ptr, S_ptr, z_ptr, stream_ptr) -> None:
@@ -185,6 +189,12 @@ def as_hybrid_attn_softmax_tokens(h, want_indices: bool = True):
 def as_hybrid_attn_last_status(h, stream_ptr) -> int:
     """Returns the status code instead of raising, so that callers can test for a time-out."""
     return lib().as_hybrid_attn_last_status(h, stream_ptr or None)
+
+
+def as_hybrid_attn_debug_expire_wait(h, limit_cycles: int, stream_ptr) -> None:
+    """Test aid: a kernel whose bounded wait runs out after `limit_cycles` SM clocks and sets the status word."""
+    _check(lib().as_hybrid_attn_debug_expire_wait(h, int(limit_cycles), stream_ptr or None),
+           "as_hybrid_attn_debug_expire_wait")
 
 
 def as_hybrid_attn_profile_enable(h, enable: bool) -> None:
@@ -212,7 +222,9 @@ def as_hybrid_attn_linear_state_static(k_ptr, v_ptr, wk_ptr, B, H, N, d, grid, b
     For callers that cannot request device memory (an arena owns all of it, or only the buffers
     handed in may be used): no handle, no workspace; the partial sums use a fixed 8 MiB array inside
     the library.  Sizes beyond that array raise AsError(AS_ERR_UNSUPPORTED).  Calls must not overlap
-    on the GPU; make the first call on a device outside any stream capture."""
+    on the GPU; make the first call on a device outside any stream capture and before an arena takes the
+    rest of the device's memory (the driver sets the array up when the library's code is first loaded on
+    the device, which by default is that first call)."""
     _check(lib().as_hybrid_attn_linear_state_static(
         k_ptr, v_ptr, wk_ptr, B, H, N, d, grid[0], grid[1], grid[2], block[0], block[1], block[2], rate,
         poly_degree, S_ptr or None, z_ptr or None, stream_ptr or None), "as_hybrid_attn_linear_state_static")

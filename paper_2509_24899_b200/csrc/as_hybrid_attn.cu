@@ -53,10 +53,17 @@ as_status_t validate(const as_hybrid_attn_desc_t* d) {
   if (d->phi_dim % d->poly_degree != 0) return AS_ERR_INVALID_ARG;
   // what the library has kernels for
   if (d->d != 64 && d->d != 128) return AS_ERR_UNSUPPORTED;
-  if (d->phi_dim != d->d) return AS_ERR_UNSUPPORTED;
-  if (d->phi_layers > 2 || d->poly_degree > 2 || d->phi_act != AS_ACT_RELU) return AS_ERR_UNSUPPORTED;
-  // two layers: hidden width equal to d, tensor-core path only
-  if (d->phi_layers == 2 && (d->phi_hidden != d->d || d->kernel_path != AS_PATH_TENSOR)) return AS_ERR_UNSUPPORTED;
+  if (d->phi_layers > 2 || d->poly_degree > 4 || d->phi_act != AS_ACT_RELU) return AS_ERR_UNSUPPORTED;
+  const int F = d->phi_dim;
+  // feature width: d itself, or a multiple of 128 up to 512; parts of the polynomial a multiple of 32 wide
+  if (!(F == d->d || (F % 128 == 0 && F <= 512))) return AS_ERR_UNSUPPORTED;
+  if ((F / d->poly_degree) % 32 != 0) return AS_ERR_UNSUPPORTED;
+  if (d->kernel_path == AS_PATH_SIMT && (F != d->d || d->phi_layers != 1 || d->poly_degree > 2)) return AS_ERR_UNSUPPORTED;
+  if (d->phi_layers == 2) {
+    // two layers: hidden width d or 2d (d = 128), features d or 2d; at d = 64 both equal to d
+    const int hid = d->phi_hidden;
+    if (d->d == 128 ? !((hid == 128 || hid == 256) && (F == 128 || F == 256)) : !(hid == 64 && F == 64)) return AS_ERR_UNSUPPORTED;
+  }
   if ((long long)d->B * d->H > 65535) return AS_ERR_UNSUPPORTED;
   return AS_OK;
 }
@@ -77,7 +84,6 @@ void layout_workspace(as_hybrid_attn_s* h) {
   w.z = take(lin ? BH * d.phi_dim * 4 : 0);
   w.Sb = take(lin ? BH * d.phi_dim * d.d * 2 : 0);
   const bool two = lin && d.phi_layers == 2;
-  w.h1q = take(two ? BH * (size_t)d.N * d.phi_hidden * 2 : 0);
   w.h1k = take(two ? BH * (size_t)d.N * d.phi_hidden * 2 : 0);
   w.total = std::max<size_t>(off, 256);
   const size_t t = BH * d.N * d.d * 2;
@@ -105,15 +111,25 @@ static as_status_t launch_heads(as_hybrid_attn_t h, const void* q, const void* k
                                 const as_phi_weights_t* w, void* out, float* aux, char* ws, cudaStream_t st,
                                 int first, int count, int nb, int nh);
 
-// The feature-map weights a layer with linear tokens needs: present, 16-byte aligned, no biases.
+// A handle works on the device it was created on: its tables live there and the kernels' shared-memory opt-in
+// was made there.
+static bool on_handle_device(const as_hybrid_attn_s* h) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return false; }
+  return dev == h->device;
+}
+
+// The feature-map weights a layer with linear tokens needs: present, 16-byte aligned; biases are optional
+// (4-byte aligned), second-layer ones only with a second layer; the fp32 check path takes none.
 static as_status_t check_weights(const as_hybrid_attn_s* h, const as_phi_weights_t* w) {
   if (h->n_l == 0) return AS_OK;
   const auto& d = h->desc;
   if (!w || !w->wq1 || !w->wk1) return AS_ERR_INVALID_ARG;
-  if (w->bq1 || w->bk1 || w->bq2 || w->bk2) return AS_ERR_UNSUPPORTED;
-  if (d.phi_layers == 1 && (w->wq2 || w->wk2)) return AS_ERR_INVALID_ARG;
+  if (d.phi_layers == 1 && (w->wq2 || w->wk2 || w->bq2 || w->bk2)) return AS_ERR_INVALID_ARG;
   if (d.phi_layers == 2 && (!w->wq2 || !w->wk2)) return AS_ERR_INVALID_ARG;
   if (((uintptr_t)w->wq1 | (uintptr_t)w->wk1 | (uintptr_t)w->wq2 | (uintptr_t)w->wk2) & 15) return AS_ERR_INVALID_ARG;
+  if (((uintptr_t)w->bq1 | (uintptr_t)w->bk1 | (uintptr_t)w->bq2 | (uintptr_t)w->bk2) & 3) return AS_ERR_INVALID_ARG;
+  if (d.kernel_path == AS_PATH_SIMT && (w->bq1 || w->bk1)) return AS_ERR_UNSUPPORTED;
   return AS_OK;
 }
 
@@ -163,14 +179,15 @@ as_status_t as_hybrid_attn_create(const as_hybrid_attn_desc_t* desc, as_hybrid_a
   int sms = 148;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int BH = desc->B * desc->H;
-  int chunks = std::max(1, std::min(tiles, sms / BH));
+  const int f_chunks = (desc->phi_dim + 127) / 128;       // the tensor K pass runs one CTA per 128 features as well
+  int chunks = std::max(1, std::min(tiles, sms / (BH * f_chunks)));
   h->chunk_tiles = (tiles + chunks - 1) / chunks;
   h->n_chunks = (tiles + h->chunk_tiles - 1) / h->chunk_tiles;
   layout_workspace(h);
 
   std::vector<int32_t> rank(desc->N, -1);
   for (int i = 0; i < h->n_s; ++i) rank[h->idx_host[i]] = i;
-  if (cudaMalloc(&h->d_sm_rank, sizeof(int32_t) * desc->N) != cudaSuccess ||
+  if (cudaMalloc(&h->d_sm_rank, sizeof(int32_t) * ((size_t)desc->N + 8)) != cudaSuccess ||
       cudaMalloc(&h->d_status, 256) != cudaSuccess) {
     cudaGetLastError(); as_hybrid_attn_destroy(h); return AS_ERR_ALLOC;
   }
@@ -226,6 +243,7 @@ as_status_t as_hybrid_attn_forward(as_hybrid_attn_t h, const void* q, const void
                                    const as_phi_weights_t* w, void* out, float* aux,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
   if (!h || !q || !k || !v || !out) return AS_ERR_INVALID_ARG;
+  if (!on_handle_device(h)) return AS_ERR_INVALID_ARG;
   const auto& d = h->desc;
   const as_status_t ws_ok = check_weights(h, w);
   if (ws_ok != AS_OK) return ws_ok;
@@ -253,14 +271,21 @@ static as_status_t launch_heads(as_hybrid_attn_t h, const void* q, const void* k
   as_launch_args a{};
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;
   const bool two = lin && d.phi_layers == 2;
-  const size_t w1 = (two ? dd : F) * dd;         // elements of one head's first-layer matrix
-  a.wq = lin ? (const __nv_bfloat16*)w->wq1 + head0 * w1 : nullptr;
-  a.wk = lin ? (const __nv_bfloat16*)w->wk1 + head0 * w1 : nullptr;
-  a.wq2 = two ? (const __nv_bfloat16*)w->wq2 + head0 * F * dd : nullptr;
-  a.wk2 = two ? (const __nv_bfloat16*)w->wk2 + head0 * F * dd : nullptr;
-  a.h1q = two ? (__nv_bfloat16*)(ws + h->ws.h1q) : nullptr;
+  const size_t hid = two ? d.phi_hidden : 0;
+  const size_t w1 = (two ? hid : F) * dd;        // elements of one head's first-layer matrix
+  const size_t b1 = two ? hid : F;               // ... and of its bias
+  auto at = [](const void* p, size_t off) { return p ? (const __nv_bfloat16*)p + off : nullptr; };
+  a.wq = lin ? at(w->wq1, head0 * w1) : nullptr;
+  a.wk = lin ? at(w->wk1, head0 * w1) : nullptr;
+  a.wq2 = two ? at(w->wq2, head0 * F * hid) : nullptr;
+  a.wk2 = two ? at(w->wk2, head0 * F * hid) : nullptr;
+  a.bq1 = lin ? at(w->bq1, head0 * b1) : nullptr;
+  a.bk1 = lin ? at(w->bk1, head0 * b1) : nullptr;
+  a.bq2 = two ? at(w->bq2, head0 * F) : nullptr;
+  a.bk2 = two ? at(w->bk2, head0 * F) : nullptr;
   a.h1k = two ? (__nv_bfloat16*)(ws + h->ws.h1k) : nullptr;
   a.layers = d.phi_layers;
+  a.hid = (int)hid;
   a.out = (__nv_bfloat16*)out; a.aux = aux;
   const bool compact = h->n_s > 0 && lin;
   a.ks_w = compact ? (__nv_bfloat16*)(ws + h->ws.ks) : nullptr;
@@ -303,6 +328,7 @@ as_status_t as_hybrid_attn_forward_host(as_hybrid_attn_t h, const void* q_host, 
                                         void* out_host, void* workspace, size_t workspace_bytes,
                                         void* cuda_stream) {
   if (!h || !q_host || !k_host || !v_host || !out_host) return AS_ERR_INVALID_ARG;
+  if (!on_handle_device(h)) return AS_ERR_INVALID_ARG;
   if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < h->ws.total_host) return AS_ERR_WORKSPACE;
   const auto& d = h->desc;
   const as_status_t ws_ok = check_weights(h, w);
@@ -364,7 +390,7 @@ as_status_t as_hybrid_attn_forward_host(as_hybrid_attn_t h, const void* q_host, 
 as_status_t as_hybrid_attn_linear_state(as_hybrid_attn_t h, const void* workspace, float* S_out,
                                         float* z_out, void* cuda_stream) {
   if (!h || !workspace) return AS_ERR_INVALID_ARG;
-  if (h->n_l == 0) return AS_ERR_INVALID_ARG;
+  if (h->n_l == 0 || !on_handle_device(h)) return AS_ERR_INVALID_ARG;
   const auto& d = h->desc;
   const size_t BH = (size_t)d.B * d.H;
   cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -379,7 +405,7 @@ as_status_t as_hybrid_attn_linear_state(as_hybrid_attn_t h, const void* workspac
 }
 
 as_status_t as_hybrid_attn_last_status(as_hybrid_attn_t h, void* cuda_stream) {
-  if (!h) return AS_ERR_INVALID_ARG;
+  if (!h || !on_handle_device(h)) return AS_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   uint32_t word = 0;
   if (cudaStreamSynchronize(st) != cudaSuccess ||
@@ -388,6 +414,15 @@ as_status_t as_hybrid_attn_last_status(as_hybrid_attn_t h, void* cuda_stream) {
   }
   if (word != 0 && cudaMemset(h->d_status, 0, 4) != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
   return (word & AS_DEV_TIMEOUT) ? AS_ERR_DEVICE_TIMEOUT : AS_OK;
+}
+
+as_status_t as_hybrid_attn_debug_expire_wait(as_hybrid_attn_t h, int64_t limit_cycles, void* cuda_stream) {
+  if (!h || !on_handle_device(h)) return AS_ERR_INVALID_ARG;
+  if (limit_cycles < 1 || limit_cycles > 100000000) return AS_ERR_INVALID_ARG;      // at most about 50 ms
+  if (as_tensor_expire_wait(h->d_status, limit_cycles, (cudaStream_t)cuda_stream) != cudaSuccess) {
+    cudaGetLastError(); return AS_ERR_CUDA;
+  }
+  return AS_OK;
 }
 
 as_status_t as_hybrid_attn_profile_enable(as_hybrid_attn_t h, int32_t enable) {

@@ -18,7 +18,7 @@ struct as_ws_layout {
   size_t part_s = 0, part_z = 0;        // per-chunk partial state   [B*H, chunks, F, d] / [.., F] fp32
   size_t S = 0, z = 0;                  // final state               [B*H, F, d] / [B*H, F] fp32
   size_t Sb = 0;                        // S rounded to bf16         [B*H, F, d] (MMA operand of the Q pass)
-  size_t h1q = 0, h1k = 0;              // first-layer activations   [B*H, N, hidden] bf16 (two-layer feature map only)
+  size_t h1k = 0;                       // first-layer activations of the keys [B*H, N, hidden] bf16 (two-layer feature map only)
   size_t total = 0;
   size_t stage_q = 0, stage_k = 0, stage_v = 0, stage_o = 0, total_host = 0;
 };
@@ -27,8 +27,10 @@ struct as_ws_layout {
 struct as_launch_args {
   const __nv_bfloat16 *q, *k, *v, *wq, *wk;
   const __nv_bfloat16 *wq2, *wk2;       // second feature-map layer [H, F, hidden] (NULL for a one-layer map)
-  __nv_bfloat16 *h1q, *h1k;             // relu(q W_q1^T), relu(k W_k1^T) when the map has two layers
+  const __nv_bfloat16 *bq1, *bk1, *bq2, *bk2;   // biases [H, width of the layer's output] (each may be NULL)
+  __nv_bfloat16* h1k;                   // relu(k W_k1^T + b_k1) [B*H, N, hidden] when the map has two layers
   int layers;                           // depth of the feature map's embedding network (1 or 2)
+  int hid;                              // hidden width of a two-layer map (0 otherwise)
   __nv_bfloat16* out;
   float* aux;
   const __nv_bfloat16 *ks, *vs;         // softmax keys / values the Q pass reads (k, v themselves at R = 1)
@@ -73,10 +75,13 @@ cudaError_t as_simt_qpass(const as_launch_args& a, cudaStream_t st);
 cudaError_t as_reduce_state(const as_launch_args& a, cudaStream_t st);
 cudaError_t as_tensor_kpass(const as_launch_args& a, cudaStream_t st);
 cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st);
-// First layer of a two-layer feature map for q and k in one launch: h1 = relu(x W1^T).
+// First layer of a two-layer feature map for the keys: h1k = relu(k W_k1^T + b_k1).
 cudaError_t as_tensor_phi1(const as_launch_args& a, cudaStream_t st);
 // One-time set-up of the tensor path on the current device (driver entry points, smem opt-in).
 cudaError_t as_tensor_init();
+
+// Test aid: a kernel whose bounded wait (the one every kernel here uses) runs out after `limit_cycles`.
+cudaError_t as_tensor_expire_wait(uint32_t* status, long long limit_cycles, cudaStream_t st);
 
 // Status bits written by kernels into as_launch_args::status.
 constexpr uint32_t AS_DEV_TIMEOUT = 1u;

@@ -16,8 +16,9 @@
 
 namespace {
 
-// Fixed scratch: 8 MiB of fp32 partial sums.  Every GPU that loads the library holds this
-// array until the process exits.
+// Fixed scratch: 8 MiB of fp32 partial sums.  A device holds this array from the moment the driver
+// loads this module there (with lazy module loading: the first call below on that device) until the
+// process exits.
 constexpr size_t kScratchFloats = size_t(2) << 20;
 static __device__ __align__(256) float g_static_scratch[kScratchFloats];
 

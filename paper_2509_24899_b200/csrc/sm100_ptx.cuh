@@ -46,7 +46,7 @@ struct WaitCtx {
 };
 constexpr long long kWaitLimitCycles = 2000ll * 1000ll * 1000ll;
 
-AS_DEV bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w) {
+AS_DEV bool mbar_wait_limit(uint32_t bar, uint32_t parity, const WaitCtx& w, long long limit_cycles) {
   if (mbar_try_wait(bar, parity)) return true;
   long long t0 = 0;
   uint32_t it = 0;
@@ -54,7 +54,7 @@ AS_DEV bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w) {
     if ((++it & 63u) == 0u) {
       const long long now = clock64();
       if (t0 == 0) t0 = now;
-      if (*w.abort != 0u || now - t0 > kWaitLimitCycles) {
+      if (*w.abort != 0u || now - t0 > limit_cycles) {
         *w.abort = 1u;
         atomicOr(w.status, 1u);
         return false;
@@ -63,6 +63,7 @@ AS_DEV bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w) {
   }
   return true;
 }
+AS_DEV bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w) { return mbar_wait_limit(bar, parity, w, kWaitLimitCycles); }
 // Warp-uniform variant: every lane waits, the result is agreed across the warp.
 AS_DEV bool mbar_wait_warp(uint32_t bar, uint32_t parity, const WaitCtx& w) {
   const bool ok = mbar_wait(bar, parity, w);

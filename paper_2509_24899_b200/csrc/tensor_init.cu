@@ -26,6 +26,31 @@ bool as_tc::make_map(CUtensorMap* m, const void* base, int cols, int rows, int s
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+namespace {
+
+// One CTA whose threads wait, with the kernels' own bounded wait, on an mbarrier that nobody arrives at.  No
+// copy and no MMA is in flight: when the limit has passed the wait gives up, raises the status bit and the
+// kernel returns.
+__global__ void expire_wait_kernel(uint32_t* status, long long limit_cycles) {
+  __shared__ uint64_t bar;
+  __shared__ uint32_t abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0u;
+    sm100::mbar_init(sm100::smem_u32(&bar), 1);
+    sm100::fence_barrier_init();
+  }
+  __syncthreads();
+  const sm100::WaitCtx wc{status, &abort_flag};
+  sm100::mbar_wait_limit(sm100::smem_u32(&bar), 0, wc, limit_cycles);
+}
+
+}  // namespace
+
+cudaError_t as_tensor_expire_wait(uint32_t* status, long long limit_cycles, cudaStream_t st) {
+  expire_wait_kernel<<<1, 64, 0, st>>>(status, limit_cycles);
+  return cudaGetLastError();
+}
+
 cudaError_t as_tensor_init() {
   std::call_once(g_once, [] {
     void* fn = nullptr;

@@ -8,9 +8,13 @@
 //                        exponentials; running max / sum per row; P = exp2(.) as bf16 -> shared memory,
 //                        O += P V_S (smem x smem -> TMEM).  Two issuing threads: one for what writes
 //                        the score columns, one for what accumulates into O.
-//   tail:                Phi = Q W_q^T -> TMEM (in the place of a next tile's scores), phi_q scaled per
-//                        row as bf16 where P sat, O += phi_q S (S in bf16 read like a V tile),
+//   tail, per chunk c of 128 features:
+//                        Phi_c = Q W_q[c]^T -> TMEM (in the place of a next tile's scores), phi_q scaled per
+//                        row as bf16 where P sat, O += phi_q,c S_c (S in bf16 read like a V tile),
 //                        den = l + phi_q.z, y = O / den -> bf16 -> staged in the P tile -> TMA store.
+//   two-layer feature map: the hidden activations relu(Q W_q1^T + b1) are formed in the same way first
+//                        (128 hidden units at a time) and kept as bf16 in the P tile and, once nothing reads
+//                        Q any more, in the Q tile; Phi_c = sum over the hidden slices of h1_j W_q2[c, j]^T.
 // All tiles are staged by TMA with the 128-byte swizzle; every mbarrier wait is bounded.
 #include "tensor_common.cuh"
 
@@ -23,7 +27,11 @@ using namespace as_tc;
 // ======================================================================================
 struct QParams {
   int N, n_s, nkv, lin, stab_mode, P, H;
-  int layers;                // depth of the feature map: with 2, tmH holds relu(q W_1^T) and tmW is W_2
+  int layers;                // depth of the feature map (1 or 2)
+  int F, fc, fcw;            // feature width, its chunks of 128 (ceil), width of a chunk (min(F, 128))
+  int nh;                    // two layers: slices of the hidden width (each D wide)
+  const __nv_bfloat16* b1;   // two layers: first-layer bias of this launch's first head [H][hidden], or nullptr
+  const __nv_bfloat16* b2;   // last-layer bias [H][F], or nullptr
   int nx, n_units;           // 256-row units per (batch, head); units over all (batch, head) pairs
   int n_rounds;              // rounds in which every CTA has a unit (n_units / gridDim.x)
   int split_last;            // 1: the units left over after those rounds are cut in two 128-row halves, one per CTA
@@ -87,31 +95,47 @@ AS_DEV int q_units_of_cta(const QParams& p) {
   return p.n_rounds + (extra ? 1 : 0);
 }
 
+// per unit and group: uses of the score columns / releases of the P tile (cf. QRing::n_s, n_pf)
+AS_DEV int q_uses_s(const QParams& p) { return p.nkv + (p.lin ? (p.layers == 2 ? p.nh + p.fc : p.fc) : 0); }
+AS_DEV int q_uses_pf(const QParams& p) { return p.nkv + (p.lin ? (p.layers == 2 ? 1 : p.fc) : 0); }
+
 template <int D>
 struct QRing {
   using L = QLayout<D>;
-  // barrier indices; per group: S (scores or Phi landed), SF (score columns read out), P (P or phi_q in
-  // shared memory), PF (the product that reads the P buffer has completed), O (output accumulator final),
-  // QF (nothing of the unit reads the Q tile any more)
+  // barrier indices; per group: S (scores, hidden activations or Phi landed in the score columns), SF (score
+  // columns read out), P (P or phi_q in shared memory), PF (the product that reads the P tile has completed),
+  // O (output accumulator final), QF (nothing of the unit reads the Q tile any more), H (two layers: the
+  // hidden activations are in shared memory)
   static constexpr int B_Q0 = 0, B_FULL = 2, B_EMPTY = B_FULL + KV_STAGES, B_S = B_EMPTY + KV_STAGES, B_SF = B_S + 2,
-                       B_P = B_SF + 2, B_PF = B_P + 2, B_O = B_PF + 2, B_QF = B_O + 2, B_COUNT = B_QF + 2;
+                       B_P = B_SF + 2, B_PF = B_P + 2, B_O = B_PF + 2, B_QF = B_O + 2, B_H = B_QF + 2, B_COUNT = B_H + 2;
   const QCtx c;              // by value: nothing here is re-read from memory after a barrier or an MMA
-  int nkv, lin, two;
-  int it_h, it_w, it_vlast, it_st, n_items, n_sp;
-  // Ring items of one unit, in the order they are consumed: K_0; then K_{j+1}, V_j for j = 0 .. nkv-2;
-  // then for the linear tail (two-layer map: the two groups' first-layer activations,) the last-layer
-  // weights; V_{nkv-1}; S in bf16.
-  AS_DEV QRing(int nkv_, int lin_, int layers, const QCtx& c_) : c(c_), nkv(nkv_), lin(lin_), two(lin_ && layers == 2) {
-    int next = nkv > 0 ? 2 * nkv - 1 : 0;
-    it_h = next; if (two) next += 2;
-    it_w = next; if (lin) next += 1;
-    it_vlast = next; if (nkv > 0) next += 1;
-    it_st = next; if (lin) next += 1;
-    n_items = next;
-    n_sp = nkv + lin;                    // per unit and group: S completions = P hand-overs = P-buffer releases
+  int nkv, lin, two, fc, nh, vl;
+  int n_stream, n_items;
+  int n_s, n_p, n_pf;        // per unit and group: uses of the score columns, P hand-overs, releases of the P tile
+  // Ring items of one unit, in the order they are consumed: K_0; then K_{j+1}, V_j for j = 0 .. nkv-2; then
+  // the linear tail with V_{nkv-1} in second place:
+  //   one layer:   W[0], V_last, then W[c], S[c-1] for c = 1 .. fc-1, then S[fc-1]
+  //   two layers:  W1[0], V_last, W1[1 .. nh-1], then W2[c, j] (c slow), then S[0 .. fc-1]
+  // addresses and waits only (the key loop needs nothing else)
+  AS_DEV explicit QRing(const QCtx& c_) : c(c_), nkv(0), lin(0), two(0), fc(0), nh(0), vl(0), n_stream(0), n_items(0), n_s(0), n_p(0), n_pf(0) {}
+  AS_DEV QRing(const QParams& p, const QCtx& c_)
+      : c(c_), nkv(p.nkv), lin(p.lin), two(p.lin && p.layers == 2), fc(p.lin ? p.fc : 0), nh(p.nh), vl(p.nkv > 0 ? 1 : 0) {
+    n_stream = nkv > 0 ? 2 * nkv - 1 : 0;
+    n_items = n_stream + vl + (two ? nh + fc * nh + fc : 2 * fc);
+    n_s = nkv + (two ? nh + fc : fc);
+    n_p = nkv + fc;
+    n_pf = nkv + (two ? 1 : fc);
   }
   AS_DEV int item_k(int j) const { return j == 0 ? 0 : 2 * j - 1; }
-  AS_DEV int item_v(int j) const { return j + 1 < nkv ? 2 * j + 2 : it_vlast; }
+  AS_DEV int it_vlast() const { return n_stream + (lin ? 1 : 0); }   // after the tail's first weight tile, if there is a tail
+  AS_DEV int item_v(int j) const { return j + 1 < nkv ? 2 * j + 2 : it_vlast(); }
+  // one layer: last-layer weights of feature chunk ch; two layers: first-layer weights of hidden slice ch
+  AS_DEV int it_w(int ch) const { return ch == 0 ? n_stream : (two ? n_stream + vl + ch : n_stream + vl + 2 * ch - 1); }
+  AS_DEV int it_w2(int ch, int j) const { return n_stream + vl + nh + ch * nh + j; }
+  AS_DEV int it_st(int ch) const {
+    if (two) return n_stream + vl + nh + fc * nh + ch;
+    return ch + 1 < fc ? n_stream + vl + 2 * ch + 2 : n_stream + vl + 2 * fc - 1;
+  }
   AS_DEV uint32_t bar(int i) const { return c.sbase + L::BAR_OFF + 8 * i; }
   AS_DEV uint32_t sQ(int g) const { return c.sbase + L::Q_OFF + g * L::TILE; }
   AS_DEV uint32_t sP(int g) const { return c.sbase + L::P_OFF + g * L::PTILE; }
@@ -138,19 +162,18 @@ struct QRing {
 };
 
 // ---------------------------------------------------------------- TMA producer, one unit
-template <int D>
+template <int D, bool TWO, bool GEN>
 __device__ __noinline__ bool q_produce_unit(const QParams& p, const QCtx& c, const CUtensorMap* tmQ, const CUtensorMap* tmK,
                                             const CUtensorMap* tmV, const CUtensorMap* tmW, const CUtensorMap* tmSt,
-                                            const CUtensorMap* tmH, int u) {
+                                            const CUtensorMap* tmW1, int u) {
   using R = QRing<D>;
   using L = QLayout<D>;
   const int nkv = p.nkv;
-  const R q(nkv, p.lin, p.layers, c);
+  const R q(p, c);
   const int lane = threadIdx.x & 31;
   const QUnit un = q_unit(p, u);
   const int bh = un.w / p.nx, h = bh % p.H, row0 = un.row0;
   const int base = u * q.n_items;
-  const int n_stream = nkv > 0 ? 2 * nkv - 1 : 0;     // K_0, then K_{j+1}, V_j alternating
   const int q_at = nkv > 0 ? 1 : 0;                   // the Q tiles are requested right after the unit's first K tile
   for (int it = 0; it < q.n_items; ++it) {
     if (it == q_at) {
@@ -168,18 +191,26 @@ __device__ __noinline__ bool q_produce_unit(const QParams& p, const QCtx& c, con
     if (!q.wait(R::B_EMPTY + st, gi / KV_STAGES + 1)) return false;
     if (lane == 0) {
       mbar_expect_tx(q.bar(R::B_FULL + st), L::TILE);
-      const uint32_t fb = q.bar(R::B_FULL + st);
-      if (it < n_stream) {
-        if (it == 0 || (it & 1)) load_tile<D>(q.sKV(gi), tmK, fb, ((it + 1) >> 1) * 128, bh);   // K_0 at 0, K_j at 2j-1
-        else load_tile<D>(q.sKV(gi), tmV, fb, ((it >> 1) - 1) * 128, bh);                        // V_j at 2j+2
-      } else if (q.two && it < q.it_w) {
-        load_tile<D>(q.sKV(gi), tmH, fb, row0 + (it - q.it_h) * 128, bh);    // relu(q W_1^T) of group it - it_h
-      } else if (q.lin && it == q.it_w) {
-        load_tile<D>(q.sKV(gi), tmW, fb, 0, h);                              // last-layer W_q[h]: [F rows][D]
-      } else if (nkv > 0 && it == q.it_vlast) {
-        load_tile<D>(q.sKV(gi), tmV, fb, (nkv - 1) * 128, bh);
+      const uint32_t fb = q.bar(R::B_FULL + st), dst = q.sKV(gi);
+      if (it < q.n_stream) {
+        if (it == 0 || (it & 1)) load_tile<D>(dst, tmK, fb, ((it + 1) >> 1) * 128, bh);   // K_0 at 0, K_j at 2j-1
+        else load_tile<D>(dst, tmV, fb, ((it >> 1) - 1) * 128, bh);                        // V_j at 2j+2
+      } else if (q.vl && it == q.it_vlast()) {
+        load_tile<D>(dst, tmV, fb, (nkv - 1) * 128, bh);
+      } else if (!TWO) {
+        // W[ch] / S[ch] in bf16: [128 feature rows][D]; rows past F arrive as zeros
+        const int r = it - q.n_stream - (it > q.n_stream ? q.vl : 0);     // 0: W[0]; 2ch-1: W[ch]; 2ch+2 (and the last): S[ch]
+        if (r == 0) load_tile<D>(dst, tmW, fb, 0, h);
+        else if (r == 2 * q.fc - 1) load_tile<D>(dst, tmSt, fb, (q.fc - 1) * 128, bh);
+        else if (r & 1) load_tile<D>(dst, tmW, fb, ((r + 1) >> 1) * 128, h);
+        else load_tile<D>(dst, tmSt, fb, ((r >> 1) - 1) * 128, bh);
       } else {
-        load_tile<D>(q.sKV(gi), tmSt, fb, 0, bh);                            // S[bh] in bf16: [F rows][D]
+        const int r = it - q.n_stream - (it > q.n_stream ? q.vl : 0);     // W1[0 .. nh-1], W2[c, j], S[c]
+        if (r < q.nh) load_tile<D>(dst, tmW1, fb, r * 128, h);                                  // hidden rows of slice r
+        else if (r < q.nh + q.fc * q.nh) {
+          const int e = r - q.nh;
+          load_boxes(dst, tmW, fb, (e % q.nh) * D, (e / q.nh) * 128, h, D / 64);                // W2[feature chunk, hidden slice]
+        } else load_tile<D>(dst, tmSt, fb, (r - q.nh - q.fc * q.nh) * 128, bh);
       }
     }
     __syncwarp();
@@ -196,15 +227,15 @@ __device__ __noinline__ bool q_produce_unit(const QParams& p, const QCtx& c, con
 // busiest resource of the CTA - every clock it spends outside the MMA instructions is a clock the tensor
 // pipe may idle - so it takes no warp votes or warp barriers, probes the barriers it needs together, and
 // has its operands ready before it looks at a barrier.
-template <int D>
+template <int D, bool TWO, bool GEN>
 __device__ __noinline__ bool q_score_unit(const QParams& p, const QCtx& c, int u) {
   using R = QRing<D>;
-  constexpr int F = D;
   constexpr uint32_t ID_QK = make_idesc(128, 128, 0, 0);      // S = Q K^T      (N = 128 keys)
-  constexpr uint32_t ID_PHI = make_idesc(128, F, 0, 0);       // Phi = Q W_q^T  (N = F)
   const int nkv = p.nkv, lin = p.lin;
-  const R q(nkv, lin, p.layers, c);
-  const int base = u * q.n_items, pb = u * q.n_sp;            // first ring item / first barrier phase of the unit
+  const R q(p, c);
+  const uint32_t id_phi = make_idesc(128, D == 128 ? 128 : p.fcw, 0, 0);   // Phi_c = X W^T  (N = features of a chunk; 128 at d = 128)
+  constexpr uint32_t ID_HID = make_idesc(128, D, 0, 0);       // hidden slice = Q W_1[j]^T (N = D hidden units)
+  const int base = u * q.n_items, ps = u * q.n_s;             // first ring item / first score-column phase of the unit
   const int ng = q_unit(p, u).ng;                             // groups at work on this unit (the last one of a group: ng - 1)
   uint64_t dq[2][8];                                          // the Q tiles do not move within a unit
 #pragma unroll
@@ -213,40 +244,14 @@ __device__ __noinline__ bool q_score_unit(const QParams& p, const QCtx& c, int u
 #pragma unroll
     for (int kk = 0; kk < 8; ++kk) dq[g][kk] = q0 + kstep_kmajor(kk);
   }
-  // Phi = X W^T with X = Q (one layer) or the first-layer activations (two layers), N = F
-  auto issue_phi = [&](int g) {
-    const uint64_t w0 = kmajor_desc(q.sKV(base + q.it_w));
-    if (q.two) {
-      const uint64_t x0 = kmajor_desc(q.sKV(base + q.it_h + g));
-#pragma unroll
-      for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), x0 + kstep_kmajor(kk), w0 + kstep_kmajor(kk), ID_PHI, kk > 0 ? 1u : 0u);
-    } else {
-#pragma unroll
-      for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), dq[g][kk], w0 + kstep_kmajor(kk), ID_PHI, kk > 0 ? 1u : 0u);
-    }
-    tc_commit(q.bar(R::B_S + g));
-    tc_commit(q.bar(R::B_QF + g));                   // nothing of this unit reads the group's Q tile any more
-    if (q.two) q.release(base + q.it_h + g);
-    if (g == ng - 1) {
-      // a lone group: the other group's first-layer tile was loaded all the same and only has to be let go
-      if (q.two && ng == 1) { q.wait_full(base + q.it_h + 1); q.release(base + q.it_h + 1); }
-      q.release(base + q.it_w);
-    }
-  };
-  // The first product of a unit overwrites score columns the previous unit's threads read last: wait for
-  // that read (the last S-free phase of the previous unit) together with the Q tile.
-  for (int g = 0; g < ng; ++g) {
-    if (u > 0 && !q.wait1(R::B_SF + g, pb - 1)) return false;
-    if (nkv == 0) {
-      if (!q.wait1(R::B_Q0 + g, u)) return false;
-      if (lin) {
-        // no softmax tokens at all: the feature product opens the unit
-        if (!q.wait_full(base + q.it_w)) return false;
-        if (q.two && !q.wait_full(base + q.it_h + g)) return false;
-        tc_fence_after();
-        issue_phi(g);
-      }
-    } else {
+  // The i-th product of the unit into a group's score columns overwrites what the threads read last: the
+  // (i-1)-th use, or the previous unit's last one.
+  auto s_free = [&](int g, int i) -> bool { return (u == 0 && i == 0) ? true : q.wait1(R::B_SF + g, ps + i - 1); };
+
+  // ---- first key tile (its product opens the unit)
+  if (nkv > 0) {
+    for (int g = 0; g < ng; ++g) {
+      if (!s_free(g, 0)) return false;
       if (!q.wait2(R::B_Q0 + g, u, g == 0, base)) return false;
       tc_fence_after();
       const uint64_t k0 = kmajor_desc(q.sKV(base));
@@ -257,43 +262,96 @@ __device__ __noinline__ bool q_score_unit(const QParams& p, const QCtx& c, int u
       if (nkv == 1 && !lin) tc_commit(q.bar(R::B_QF + g));
     }
   }
-  for (int j = 0; j < nkv; ++j) {
-    const bool last = (j + 1 == nkv);
-    // as soon as the groups have read their score rows: the next tile's Q K^T, or Phi after the last tile
-    if (!last) {
-      const int ik = base + q.item_k(j + 1);
-      const uint64_t k0 = kmajor_desc(q.sKV(ik));
+  // ---- as soon as the groups have read their score rows: the next tile's Q K^T
+  for (int j = 0; j + 1 < nkv; ++j) {
+    const int ik = base + q.item_k(j + 1);
+    const uint64_t k0 = kmajor_desc(q.sKV(ik));
 #pragma unroll
-      for (int g = 0; g < 2; ++g) {
-        if (g >= ng) break;
-        if (!q.wait2(R::B_SF + g, pb + j, g == 0, ik)) return false;
-        tc_fence_after();
+    for (int g = 0; g < 2; ++g) {
+      if (g >= ng) break;
+      if (!q.wait2(R::B_SF + g, ps + j, g == 0, ik)) return false;
+      tc_fence_after();
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), dq[g][kk], k0 + kstep_kmajor(kk), ID_QK, kk > 0 ? 1u : 0u);
-        tc_commit(q.bar(R::B_S + g));
-        if (j + 2 == nkv && !lin) tc_commit(q.bar(R::B_QF + g));   // the unit's last read of the Q tile
-      }
-      q.release(ik);
-    } else if (lin) {
+      for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), dq[g][kk], k0 + kstep_kmajor(kk), ID_QK, kk > 0 ? 1u : 0u);
+      tc_commit(q.bar(R::B_S + g));
+      if (j + 2 == nkv && !lin) tc_commit(q.bar(R::B_QF + g));   // the unit's last read of the Q tile
+    }
+    q.release(ik);
+  }
+  if (!lin) return true;
+
+  // ---- linear tail: what lands in the score columns after the last key tile
+  if constexpr (!TWO) {
+    // Phi_c = Q W[c]^T, one chunk of features after the other
+    for (int ch = 0; ch < q.fc; ++ch) {
+      const int iw = base + q.it_w(ch);
+      const uint64_t w0 = kmajor_desc(q.sKV(iw));
       for (int g = 0; g < ng; ++g) {
-        if (!q.wait2(R::B_SF + g, pb + j, g == 0, base + q.it_w)) return false;
-        if (q.two && !q.wait_full(base + q.it_h + g)) return false;
+        if (!s_free(g, nkv + ch)) return false;
+        if (nkv == 0 && ch == 0 && !q.wait1(R::B_Q0 + g, u)) return false;
+        if (g == 0 && !q.wait_full(iw)) return false;
         tc_fence_after();
-        issue_phi(g);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), dq[g][kk], w0 + kstep_kmajor(kk), id_phi, kk > 0 ? 1u : 0u);
+        tc_commit(q.bar(R::B_S + g));
+        if (ch == q.fc - 1) tc_commit(q.bar(R::B_QF + g));     // nothing of this unit reads the group's Q tile any more
       }
+      q.release(iw);
+    }
+    return true;
+  } else {
+  // two layers: hidden slices first (A = Q), then Phi_c = sum_j h1_j W2[c, j]^T with the hidden slices read from
+  // where the threads put them: slice 0 in the group's P tile, slice 1 in its Q tile
+  for (int j = 0; j < q.nh; ++j) {
+    const int iw = base + q.it_w(j);
+    const uint64_t w0 = kmajor_desc(q.sKV(iw));
+    for (int g = 0; g < ng; ++g) {
+      if (!s_free(g, nkv + j)) return false;
+      if (nkv == 0 && j == 0 && !q.wait1(R::B_Q0 + g, u)) return false;
+      if (g == 0 && !q.wait_full(iw)) return false;
+      tc_fence_after();
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) mma_ss(q.tS(g), dq[g][kk], w0 + kstep_kmajor(kk), ID_HID, kk > 0 ? 1u : 0u);
+      tc_commit(q.bar(R::B_S + g));
+      if (q.nh == 1 && q.fc == 1) tc_commit(q.bar(R::B_QF + g));   // the Q tile is not reused as a buffer in this shape
+    }
+    q.release(iw);
+  }
+  for (int ch = 0; ch < q.fc; ++ch) {
+    for (int j = 0; j < q.nh; ++j) {
+      const int iw = base + q.it_w2(ch, j);
+      const uint64_t w0 = kmajor_desc(q.sKV(iw));
+      if (!q.wait_full(iw)) return false;
+      for (int g = 0; g < ng; ++g) {
+        if (j == 0) {
+          if (!s_free(g, nkv + q.nh + ch)) return false;
+          if (ch == 0 && !q.wait1(R::B_H + g, u)) return false;   // the group's hidden activations are in shared memory
+        }
+        tc_fence_after();
+        const uint64_t a0 = kmajor_desc(j == 0 ? q.sP(g) : q.sQ(g));
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk)
+          mma_ss(q.tS(g), a0 + kstep_kmajor(kk), w0 + kstep_kmajor(kk), id_phi, (j > 0 || kk > 0) ? 1u : 0u);
+        if (j == q.nh - 1) {
+          tc_commit(q.bar(R::B_S + g));
+          // two hidden slices, one feature chunk: this was the last read of the Q tile (as a buffer)
+          if (q.nh == 2 && q.fc == 1) tc_commit(q.bar(R::B_QF + g));
+        }
+      }
+      q.release(iw);
     }
   }
   return true;
+  }
 }
 
-template <int D>
+template <int D, bool TWO, bool GEN>
 __device__ __noinline__ bool q_accum_unit(const QParams& p, const QCtx& c, int u) {
   using R = QRing<D>;
-  constexpr int F = D;
   constexpr uint32_t ID_PV = make_idesc(128, D, 0, 1);        // O += P V and O += phi_q S  (V, S are MN-major)
   const int nkv = p.nkv, lin = p.lin;
-  const R q(nkv, lin, p.layers, c);
-  const int base = u * q.n_items, pb = u * q.n_sp;            // first ring item / first barrier phase of the unit
+  const R q(p, c);
+  const int base = u * q.n_items, pp = u * q.n_p;             // first ring item / first P hand-over phase of the unit
   const int ng = q_unit(p, u).ng;
   uint64_t dp[2][8];                                          // the P tiles never move
 #pragma unroll
@@ -310,7 +368,7 @@ __device__ __noinline__ bool q_accum_unit(const QParams& p, const QCtx& c, int u
 #pragma unroll
     for (int g = 0; g < 2; ++g) {
       if (g >= ng) break;
-      if (!q.wait2(R::B_P + g, pb + j, g == 0, iv)) return false;
+      if (!q.wait2(R::B_P + g, pp + j, g == 0, iv)) return false;
       tc_fence_after();
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) mma_ss(q.tO(g), dp[g][kk], v0 + kstep_mnmajor(kk), ID_PV, (j > 0 || kk > 0) ? 1u : 0u);
@@ -319,39 +377,216 @@ __device__ __noinline__ bool q_accum_unit(const QParams& p, const QCtx& c, int u
     }
     q.release(iv);
   }
-  if (lin) {
-    const int is = base + q.it_st;
+  if (!lin) return true;
+  // O += phi_q,c S_c per feature chunk: phi_q sits where P sits (two layers, second chunk: in the Q tile),
+  // S plays the part of a V tile
+  const int ksteps = (D == 128 ? 128 : p.fcw) / 16;           // a constant at d = 128: the chains below unroll
+  for (int ch = 0; ch < q.fc; ++ch) {
+    const int is = base + q.it_st(ch);
     const uint64_t s0 = mnmajor_desc(q.sKV(is));
+    const bool in_q_tile = TWO && ch == 1;
     for (int g = 0; g < ng; ++g) {
-      if (!q.wait2(R::B_P + g, pb + nkv, g == 0, is)) return false;
+      if (!q.wait2(R::B_P + g, pp + nkv + ch, g == 0, is)) return false;
       tc_fence_after();
-      // phi_q sits where P sits, S plays the part of a V tile
+      const uint64_t a0 = in_q_tile ? kmajor_desc(q.sQ(g)) : dp[g][0];
 #pragma unroll
-      for (int kk = 0; kk < F / 16; ++kk) mma_ss(q.tO(g), dp[g][kk], s0 + kstep_mnmajor(kk), ID_PV, (nkv > 0 || kk > 0) ? 1u : 0u);
-      tc_commit(q.bar(R::B_PF + g));
-      tc_commit(q.bar(R::B_O + g));
-      if (g == ng - 1) q.release(is);
+      for (int kk = 0; kk < 8; ++kk)
+        if (kk < ksteps) mma_ss(q.tO(g), a0 + kstep_kmajor(kk), s0 + kstep_mnmajor(kk), ID_PV, (nkv > 0 || ch > 0 || kk > 0) ? 1u : 0u);
+      if (!in_q_tile) tc_commit(q.bar(R::B_PF + g));           // a reader of the P tile has completed
+      if (ch == q.fc - 1) {
+        tc_commit(q.bar(R::B_O + g));
+        if (in_q_tile) tc_commit(q.bar(R::B_QF + g));          // ... and the last reader of the Q tile
+      }
     }
+    q.release(is);
   }
   return true;
 }
 
-// ---------------------------------------------------------------- softmax / merge group, one unit
+// ---------------------------------------------------------------- feature rows of the linear tail
+// One row of Phi (feature chunk ch), already read out of the score columns into ph -> bf16(lam * poly(relu(Phi + b)))
+// -> row r of `tile` (the A operand of the apply product).  Returns the row's share of phi_q.z, formed with the very
+// bf16 values the MMA multiplies with S.  GEN = false is the common case (no bias, polynomial degree <= 2).
+template <int D, bool GEN>
+AS_DEV float q_features_to_tile(const QParams& p, const uint32_t (&ph)[128], uint8_t* tile, int r, int bh, int ch, float lam) {
+  const int fcw = D == 128 ? 128 : p.fcw;            // a chunk is narrower than 128 only at d = F = 64
+  const int part = p.F / p.P;
+  const float2* zrow = reinterpret_cast<const float2*>(p.z + (size_t)bh * p.F + ch * 128);
+  const uint32_t* brow = nullptr;
+  if (GEN && p.b2 != nullptr) brow = reinterpret_cast<const uint32_t*>(p.b2 + (size_t)(bh % p.H) * p.F + ch * 128);
+  float dl0 = 0.f, dl1 = 0.f;
+#pragma unroll
+  for (int cc = 0; cc < 4; ++cc) {
+    if (cc * 32 < fcw) {
+      const int pw = min((ch * 128 + cc * 32) / part, p.P - 1);     // 0-based part of these 32 features
+      uint32_t wd[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        float a0 = __uint_as_float(ph[cc * 32 + 2 * i]), a1 = __uint_as_float(ph[cc * 32 + 2 * i + 1]);
+        if (GEN && brow != nullptr) {
+          const uint32_t bb = __ldg(brow + cc * 16 + i);            // same address in every lane: one broadcast load
+          a0 += __uint_as_float(bb << 16);
+          a1 += __uint_as_float(bb & 0xffff0000u);
+        }
+        a0 = fmaxf(a0, 0.f); a1 = fmaxf(a1, 0.f);
+        float r0 = a0, r1 = a1;
+        if (pw >= 1) { r0 *= a0; r1 *= a1; }
+        if (GEN) {
+          if (pw >= 2) { r0 *= a0; r1 *= a1; }
+          if (pw >= 3) { r0 *= a0; r1 *= a1; }
+        }
+        wd[i] = pack_bf16(r0 * lam, r1 * lam);
+        const float2 zz = __ldg(zrow + cc * 16 + i);
+        dl0 = fmaf(__uint_as_float(wd[i] << 16), zz.x, dl0);
+        dl1 = fmaf(__uint_as_float(wd[i] & 0xffff0000u), zz.y, dl1);
+      }
+      store_row_chunk(tile, r, cc * 32, wd);
+    }
+  }
+  fence_proxy_async();
+  return dl0 + dl1;
+}
+
+// Reads one row of the score columns (ncols of them) at once and releases the columns.
 template <int D>
+AS_DEV void q_read_row(const QRing<D>& q, int g, uint32_t tSg, int ncols, uint32_t (&ph)[128]) {
+  using R = QRing<D>;
+  uint32_t x[32];
+#pragma unroll
+  for (int cc = 0; cc < 4; ++cc) {
+    if (cc * 32 < ncols) {
+      tmem_ld32(tSg + cc * 32, x);
+      tmem_ld_wait(x);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) ph[cc * 32 + i] = x[i];
+    }
+  }
+  tc_fence_before();
+  mbar_arrive(q.bar(R::B_SF + g));                   // the next product into the score columns may follow
+}
+
+// Two-layer feature map, one unit and group: hidden slices relu(Q W_1[j]^T + b_1) as bf16 (slice 0 into the P tile,
+// slice 1 into the Q tile, free once the product that made slice 1, the last reader of Q, has completed), then the
+// feature chunks.  Returns phi_q.z, or -1 when a wait ran out.
+template <int D, bool GEN>
+__device__ __noinline__ float q_two_layer_tail(const QParams& p, const QRing<D>& q, int g, uint32_t tSg, uint8_t* sPg, uint8_t* sQg,
+                                               int r, int bh, int ps, int ppf, float lam) {
+  using R = QRing<D>;
+  const int nkv = p.nkv, h = bh % p.H, lane = threadIdx.x & 31;
+  const __nv_bfloat16* b1 = (GEN && p.b1) ? p.b1 + (size_t)h * (q.nh * D) : nullptr;
+  uint32_t x[32];
+  for (int j = 0; j < q.nh; ++j) {
+    if (!q.wait(R::B_S + g, ps + nkv + j)) return -1.f;
+    tc_fence_after();
+    if (j == 0) {                                    // the last tile's P V has read the P tile (cf. the key loop)
+      if (lane == 0) tma_store_wait_read();
+      if (ppf + nkv == 0) __syncwarp();
+      else if (!q.wait(R::B_PF + g, ppf + nkv - 1)) return -1.f;
+    }
+    const uint32_t* brow = b1 ? reinterpret_cast<const uint32_t*>(b1 + j * D) : nullptr;
+    uint8_t* tile = j == 0 ? sPg : sQg;
+#pragma unroll
+    for (int cc = 0; cc < D / 32; ++cc) {
+      tmem_ld32(tSg + cc * 32, x);
+      tmem_ld_wait(x);
+      uint32_t wd[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        float a0 = __uint_as_float(x[2 * i]), a1 = __uint_as_float(x[2 * i + 1]);
+        if (brow != nullptr) {
+          const uint32_t bb = __ldg(brow + cc * 16 + i);
+          a0 += __uint_as_float(bb << 16);
+          a1 += __uint_as_float(bb & 0xffff0000u);
+        }
+        wd[i] = pack_bf16(fmaxf(a0, 0.f), fmaxf(a1, 0.f));
+      }
+      store_row_chunk(tile, r, cc * 32, wd);
+    }
+    tc_fence_before();
+    mbar_arrive(q.bar(R::B_SF + g));
+    fence_proxy_async();
+    mbar_arrive(q.bar(R::B_H + g));
+  }
+  // Feature chunks.  The hidden slices stay in their buffers until the last chunk's product has completed, so with
+  // two chunks the first one's features wait in shared memory nobody else uses at that time: the rows of the group's
+  // P tile are still the hidden slice, but ... (see below)
+  if (!q.wait(R::B_S + g, ps + nkv + q.nh)) return -1.f;
+  tc_fence_after();
+  if (q.fc == 1) {
+    uint32_t ph[128];
+    q_read_row<D>(q, g, tSg, D == 128 ? 128 : p.fcw, ph);
+    const float dl = q_features_to_tile<D, GEN>(p, ph, sPg, r, bh, 0, lam);   // Phi_0 is complete: nothing reads the slices any more
+    mbar_arrive(q.bar(R::B_P + g));
+    return dl;
+  }
+  // two chunks: chunk 0 is kept as bf16 pairs in registers until Phi_1 has landed (then the slices are free)
+  float dl0 = 0.f, dl1 = 0.f;
+  uint32_t pk[64];
+  {
+    const int part = p.F / p.P;
+    const float2* zrow = reinterpret_cast<const float2*>(p.z + (size_t)bh * p.F);
+    const uint32_t* brow = (GEN && p.b2) ? reinterpret_cast<const uint32_t*>(p.b2 + (size_t)h * p.F) : nullptr;
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+      tmem_ld32(tSg + cc * 32, x);
+      tmem_ld_wait(x);
+      const int pw = min((cc * 32) / part, p.P - 1);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        float a0 = __uint_as_float(x[2 * i]), a1 = __uint_as_float(x[2 * i + 1]);
+        if (brow != nullptr) {
+          const uint32_t bb = __ldg(brow + cc * 16 + i);
+          a0 += __uint_as_float(bb << 16);
+          a1 += __uint_as_float(bb & 0xffff0000u);
+        }
+        a0 = fmaxf(a0, 0.f); a1 = fmaxf(a1, 0.f);
+        float r0 = a0, r1 = a1;
+        if (pw >= 1) { r0 *= a0; r1 *= a1; }
+        if (pw >= 2) { r0 *= a0; r1 *= a1; }
+        if (pw >= 3) { r0 *= a0; r1 *= a1; }
+        const uint32_t wv = pack_bf16(r0 * lam, r1 * lam);
+        pk[cc * 16 + i] = wv;
+        const float2 zz = __ldg(zrow + cc * 16 + i);
+        dl0 = fmaf(__uint_as_float(wv << 16), zz.x, dl0);
+        dl1 = fmaf(__uint_as_float(wv & 0xffff0000u), zz.y, dl1);
+      }
+    }
+    tc_fence_before();
+    mbar_arrive(q.bar(R::B_SF + g));                 // Phi_1 may overwrite the score columns
+  }
+  if (!q.wait(R::B_S + g, ps + nkv + q.nh + 1)) return -1.f;     // Phi_1 is there: nothing reads the hidden slices any more
+  tc_fence_after();
+#pragma unroll
+  for (int cc = 0; cc < 4; ++cc) {
+    uint32_t wd[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) wd[i] = pk[cc * 16 + i];
+    store_row_chunk(sPg, r, cc * 32, wd);
+  }
+  fence_proxy_async();
+  mbar_arrive(q.bar(R::B_P + g));
+  uint32_t ph[128];
+  q_read_row<D>(q, g, tSg, 128, ph);
+  const float dlb = q_features_to_tile<D, GEN>(p, ph, sQg, r, bh, 1, lam);
+  mbar_arrive(q.bar(R::B_P + g));
+  return (dl0 + dl1) + dlb;
+}
+
+// ---------------------------------------------------------------- softmax / merge group, one unit
+template <int D, bool TWO, bool GEN>
 __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, const CUtensorMap* tmO, uint8_t* smem, int u) {
   using R = QRing<D>;
   using L = QLayout<D>;
-  constexpr int F = D;
   const int nkv = p.nkv, n_s = p.n_s;
   const float scale_log2 = p.scale_log2;
-  const R q(nkv, p.lin, p.layers, c);
+  const R q(p, c);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = warp >> 2;                          // group 0 or 1
   const int r = (warp & 3) * 32 + lane;             // row inside the group's 128-row tile
   const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
   const uint32_t tSg = q.tS(g) + lane_off, tOg = q.tO(g) + lane_off;
   uint8_t* sPg = smem + L::P_OFF + g * L::PTILE;    // this group's P / phi_q / output staging tile
-  const int pb = u * q.n_sp;
+  const int ps = u * q.n_s, ppf = u * q.n_pf;       // first phases of the unit (cf. QRing)
   float m_ref = 0.f, m_true = -INFINITY, l = 0.f;
   uint32_t x[32];
 
@@ -364,7 +599,7 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
   };
 
   for (int j = 0; j < nkv; ++j) {
-    if (!q.wait(R::B_S + g, pb + j)) return false;
+    if (!q.wait(R::B_S + g, ps + j)) return false;
     tc_fence_after();
     uint32_t sv[128];                               // this thread's row of the 128 x 128 score tile
     tmem_ld128_sync(tSg, sv);
@@ -409,7 +644,7 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
         pw[2 * i] = pack_bf16(pa.x, pa.y);
         pw[2 * i + 1] = pack_bf16(pc.x, pc.y);
       }
-      if (cc == 0 && !p_buffer_free(pb + j)) return false;   // the previous tile's P V has read the buffer
+      if (cc == 0 && !p_buffer_free(ppf + j)) return false;  // the previous tile's P V has read the buffer
       store_row_chunk(sPg, r, cc * 32, pw);
     }
     // The sum above adds the unrounded probabilities while the MMA multiplies their bf16 roundings with V.
@@ -447,41 +682,24 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
     if (nkv > 0) e = (p.stab_mode == AS_STAB_EXACT) ? -m_ref : (m_true - m_ref);
     e = fminf(fmaxf(e, -100.f), 100.f);
     const float lam = ex2(e);
-    const float2* zrow = reinterpret_cast<const float2*>(p.z + (size_t)bh * F);
-    if (!q.wait(R::B_S + g, pb + nkv)) return false;
-    tc_fence_after();
-    uint32_t ph[F];                                  // this thread's row of Phi: read at once, columns released
-    float dl0 = 0.f, dl1 = 0.f;
-    const bool two_parts = (p.P == 2);
-#pragma unroll
-    for (int cc = 0; cc < F / 32; ++cc) {
-      tmem_ld32(tSg + cc * 32, x);
-      tmem_ld_wait(x);
-#pragma unroll
-      for (int i = 0; i < 32; ++i) ph[cc * 32 + i] = x[i];
-    }
-    tc_fence_before();
-    mbar_arrive(q.bar(R::B_SF + g));                 // the next unit's first Q K^T may overwrite the columns
-    if (!p_buffer_free(pb + nkv)) return false;      // the last tile's P V has read the buffer
-#pragma unroll
-    for (int cc = 0; cc < F / 32; ++cc) {
-      const bool squared = two_parts && (cc * 32 >= F / 2);
-      uint32_t wd[16];
-#pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        float a0 = fmaxf(__uint_as_float(ph[cc * 32 + 2 * i]), 0.f), a1 = fmaxf(__uint_as_float(ph[cc * 32 + 2 * i + 1]), 0.f);
-        if (squared) { a0 *= a0; a1 *= a1; }
-        wd[i] = pack_bf16(a0 * lam, a1 * lam);
-        // the denominator uses the very bf16 values the MMA multiplies with S
-        const float2 zz = __ldg(zrow + cc * 16 + i);   // same address in every lane: one broadcast load
-        dl0 = fmaf(__uint_as_float(wd[i] << 16), zz.x, dl0);
-        dl1 = fmaf(__uint_as_float(wd[i] & 0xffff0000u), zz.y, dl1);
+    float dl;
+    dl = 0.f;
+    if constexpr (!TWO) {
+      for (int ch = 0; ch < q.fc; ++ch) {
+        if (!q.wait(R::B_S + g, ps + nkv + ch)) return false;
+        tc_fence_after();
+        uint32_t ph[128];                              // this thread's row of Phi: read at once, columns released
+        q_read_row<D>(q, g, tSg, D == 128 ? 128 : p.fcw, ph);
+        if (!p_buffer_free(ppf + nkv + ch)) return false;   // the last tile's P V / the previous chunk's product has read the P tile
+        dl += q_features_to_tile<D, GEN>(p, ph, sPg, r, bh, ch, lam);     // phi_q takes P's place as the A operand
+        mbar_arrive(q.bar(R::B_P + g));
       }
-      store_row_chunk(sPg, r, cc * 32, wd);          // phi_q takes P's place as the A operand
     }
-    const float dl = dl0 + dl1;
-    fence_proxy_async();
-    mbar_arrive(q.bar(R::B_P + g));
+    if constexpr (TWO) {
+      uint8_t* sQg = smem + L::Q_OFF + g * L::TILE;    // the group's Q tile: a second buffer once Q is done with
+      dl = q_two_layer_tail<D, GEN>(p, q, g, tSg, sPg, sQg, r, bh, ps, ppf, lam);
+      if (dl < 0.f) return false;                      // a wait ran out (the sum itself is never negative)
+    }
     den = l + dl;
     den_l_out = dl / lam;
   }
@@ -522,11 +740,11 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
   return true;
 }
 
-template <int D>
+template <int D, bool TWO, bool GEN>
 __global__ void __launch_bounds__(Q_THREADS, 1)
 qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
              const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmW,
-             const __grid_constant__ CUtensorMap tmSt, const __grid_constant__ CUtensorMap tmH,
+             const __grid_constant__ CUtensorMap tmSt, const __grid_constant__ CUtensorMap tmW1,
              const __grid_constant__ CUtensorMap tmO, const __grid_constant__ QParams p) {
   using L = QLayout<D>;
   using R = QRing<D>;
@@ -551,6 +769,7 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     for (int g = 0; g < 2; ++g) {
       mbar_init(bar(R::B_S + g), 1); mbar_init(bar(R::B_SF + g), 128); mbar_init(bar(R::B_P + g), 128);
       mbar_init(bar(R::B_PF + g), 1); mbar_init(bar(R::B_O + g), 1); mbar_init(bar(R::B_QF + g), 1);
+      mbar_init(bar(R::B_H + g), 128 * (p.nh > 0 ? p.nh : 1));   // one arrival per thread and hidden slice
     }
     fence_barrier_init();
     fence_proxy_async();
@@ -565,24 +784,24 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   if (warp == 8) {
     if ((threadIdx.x & 31) == 0) { tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmO); }
     for (int u = 0; u < n_mine; ++u)
-      if (!q_produce_unit<D>(p, c, &tmQ, &tmK, &tmV, &tmW, &tmSt, &tmH, u)) break;
+      if (!q_produce_unit<D, TWO, GEN>(p, c, &tmQ, &tmK, &tmV, &tmW, &tmSt, &tmW1, u)) break;
   } else if (warp == 9) {
     if ((threadIdx.x & 31) == 0) {
       for (int u = 0; u < n_mine; ++u)
-        if (!q_score_unit<D>(p, c, u)) break;
+        if (!q_score_unit<D, TWO, GEN>(p, c, u)) break;
     }
     __syncwarp();
   } else if (warp == 10) {
     if ((threadIdx.x & 31) == 0) {
       for (int u = 0; u < n_mine; ++u)
-        if (!q_accum_unit<D>(p, c, u)) break;
+        if (!q_accum_unit<D, TWO, GEN>(p, c, u)) break;
     }
     __syncwarp();
   } else {
     // a unit worked on by one group only (a left-over half) is the CTA's last one: group 1 stops before it
     const int n_grp = (n_mine > p.n_rounds && p.split_last && warp >= 4) ? p.n_rounds : n_mine;
     for (int u = 0; u < n_grp; ++u)
-      if (!q_softmax_unit<D>(p, c, &tmO, smem, u)) break;
+      if (!q_softmax_unit<D, TWO, GEN>(p, c, &tmO, smem, u)) break;
     if ((threadIdx.x & 31) == 0) tma_store_wait_all();   // this warp's output stores have completed
   }
 
@@ -599,15 +818,21 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 
 cudaError_t as_tensor_init_qpass() {
   cudaError_t e;
-  if ((e = opt_in_smem(qpass_kernel<128>, QLayout<128>::TOTAL)) != cudaSuccess) return e;
-  if ((e = opt_in_smem(qpass_kernel<64>, QLayout<64>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(qpass_kernel<128, false, false>, QLayout<128>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(qpass_kernel<128, false, true>, QLayout<128>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(qpass_kernel<128, true, false>, QLayout<128>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(qpass_kernel<128, true, true>, QLayout<128>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(qpass_kernel<64, false, false>, QLayout<64>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(qpass_kernel<64, false, true>, QLayout<64>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(qpass_kernel<64, true, false>, QLayout<64>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(qpass_kernel<64, true, true>, QLayout<64>::TOTAL)) != cudaSuccess) return e;
   return cudaSuccess;
 }
 
 cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st) {
   const int BH = a.B * a.H;
   const bool lin = a.n_l > 0;
-  CUtensorMap tmQ, tmK, tmV, tmW, tmSt, tmH, tmO;
+  CUtensorMap tmQ, tmK, tmV, tmW, tmSt, tmW1, tmO;
   // the output is stored warp by warp: boxes of 32 rows
   if (!make_map(&tmQ, a.q, a.d, a.N, BH, 128) || !make_map(&tmO, a.out, a.d, a.N, BH, 32)) return cudaErrorInvalidValue;
   if (a.n_s > 0) {
@@ -615,18 +840,25 @@ cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st) {
   } else {
     tmK = tmQ; tmV = tmQ;       // never used: the key loop is empty
   }
+  const bool two = lin && a.layers == 2;
   if (lin) {
-    // boxes are always 128 rows: rows past F (or d) are out of bounds and arrive as zeros
-    if (!make_map(&tmW, a.layers == 2 ? a.wq2 : a.wq, a.d, a.F, a.H, 128) || !make_map(&tmSt, a.Sb, a.d, a.F, BH, 128)) return cudaErrorInvalidValue;
+    // boxes are always 128 rows: rows past F (or the hidden width) are out of bounds and arrive as zeros.
+    // tmW: last-layer weights [H][F][width of their input]; tmW1: first-layer weights of a two-layer map.
+    if (!make_map(&tmW, two ? a.wq2 : a.wq, two ? a.hid : a.d, a.F, a.H, 128) || !make_map(&tmSt, a.Sb, a.d, a.F, BH, 128))
+      return cudaErrorInvalidValue;
   } else {
     tmW = tmQ; tmSt = tmQ;      // never used: no linear branch at rate 1
   }
-  if (lin && a.layers == 2) { if (!make_map(&tmH, a.h1q, a.d, a.N, BH, 128)) return cudaErrorInvalidValue; }
-  else tmH = tmQ;             // never used with a one-layer map
+  if (two) { if (!make_map(&tmW1, a.wq, a.d, a.hid, a.H, 128)) return cudaErrorInvalidValue; }
+  else tmW1 = tmQ;            // never used with a one-layer map
   QParams p{};
   p.layers = lin ? a.layers : 1;
   p.N = a.N; p.n_s = a.n_s; p.nkv = (a.n_s + 127) / 128; p.lin = lin ? 1 : 0; p.stab_mode = a.stab_mode; p.P = a.P;
   p.H = a.H;
+  p.F = a.F; p.fc = (a.F + 127) / 128; p.fcw = a.F < 128 ? a.F : 128;
+  p.nh = two ? a.hid / a.d : 0;
+  p.b1 = two ? a.bq1 : nullptr;
+  p.b2 = two ? a.bq2 : a.bq1;
   p.scale_log2 = a.scale * 1.4426950408889634f;
   p.z = a.z; p.aux = a.aux; p.status = a.status;
   p.nx = (a.N + 255) / 256;
@@ -640,7 +872,17 @@ cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st) {
   const int left = p.n_units - p.n_rounds * (int)grid.x;
   // left-over units as 128-row halves when twice their number still fits the grid
   p.split_last = (left > 0 && 2 * left <= (int)grid.x) ? 1 : 0;
-  if (a.d == 128) qpass_kernel<128><<<grid, Q_THREADS, QLayout<128>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmH, tmO, p);
-  else qpass_kernel<64><<<grid, Q_THREADS, QLayout<64>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmH, tmO, p);
+  // the general kernels carry the bias and the powers beyond 2; the common case does without them
+  const bool gen = lin && (a.P > 2 || p.b1 != nullptr || p.b2 != nullptr);
+#define AS_LAUNCH_Q(D_, TWO_, GEN_) \
+  qpass_kernel<D_, TWO_, GEN_><<<grid, Q_THREADS, QLayout<D_>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmW1, tmO, p)
+  if (a.d == 128) {
+    if (two) { if (gen) AS_LAUNCH_Q(128, true, true); else AS_LAUNCH_Q(128, true, false); }
+    else { if (gen) AS_LAUNCH_Q(128, false, true); else AS_LAUNCH_Q(128, false, false); }
+  } else {
+    if (two) { if (gen) AS_LAUNCH_Q(64, true, true); else AS_LAUNCH_Q(64, true, false); }
+    else { if (gen) AS_LAUNCH_Q(64, false, true); else AS_LAUNCH_Q(64, false, false); }
+  }
+#undef AS_LAUNCH_Q
   return cudaGetLastError();
 }

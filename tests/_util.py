@@ -131,13 +131,25 @@ def oracle_mask(wl):
     return O.softmax_token_mask(wl.grid, wl.block, wl.rate)
 
 
+def head_weights(data64, which, h):
+    """The oracle's view of one head's feature map: a matrix, or a list of layers, each a matrix or a
+    (matrix, bias) pair.  `which` is "q" or "k"; data64 holds wq/wk (, wq2/wk2) (, bq1/bk1, bq2/bk2)."""
+    def layer(wname, bname):
+        Wm = data64[wname][h]
+        return (Wm, data64[bname][h]) if bname in data64 else Wm
+    first = layer("w" + which, "b" + which + "1")
+    if ("w" + which + "2") not in data64:
+        return first if not isinstance(first, tuple) else [first]
+    return [first, layer("w" + which + "2", "b" + which + "2")]
+
+
 def balanced_gain(wl, stab_mode, sample_rows=48, seed=123):
-    """Gain g for W_q such that the median over sampled queries of lambda_i*den_L/den_S is 1.
+    """Gain g for the query feature map such that the median over sampled queries of lambda_i*den_L/den_S is 1.
 
     With Glorot-random feature maps the linear branch outweighs the softmax branch by orders of
-    magnitude, and a wrong softmax branch would hide inside the tolerance.  Scaling W_q by g
-    (before bf16 rounding, as the generator does) makes both branches matter.  Uses the oracle only.
-    """
+    magnitude, and a wrong softmax branch would hide inside the tolerance.  Scaling the last layer of the
+    query map by g (before bf16 rounding, as the generator does) makes both branches matter.  Uses the
+    oracle only."""
     mask = oracle_mask(wl)
     if mask.all() or not mask.any():
         return 1.0
@@ -145,22 +157,21 @@ def balanced_gain(wl, stab_mode, sample_rows=48, seed=123):
     rng = np.random.default_rng(seed)
     rows = np.sort(rng.choice(wl.N, size=min(sample_rows, wl.N), replace=False))
     q, k, v = data["q"][0, 0], data["k"][0, 0], data["v"][0, 0]
-    _, z = O.linear_state(k, v, data["wk"][0], mask, wl.degree)
+    _, z = O.linear_state(k, v, head_weights(data, "k", 0), mask, wl.degree)
     s = (q[rows] @ k[mask].T) / math.sqrt(wl.d)
     c = s.max(1)
     den_s = np.exp(s - c[:, None]).sum(1)
     lam = np.exp(-c) if stab_mode == O.STAB_EXACT else np.ones_like(c)
-    wq32 = W.bf16_bits_to_f32(W.generate(wl, heads=1)["wq"][0])     # gain-1 weights (bf16 values)
 
     def ratio(g):
-        wq = W.bf16_bits_to_f64(W.f32_to_bf16_bits(wq32 * np.float32(g)))
-        den_l = O.phi_features(q[rows], wq, wl.degree) @ z
+        dg = oracle_inputs({n: a for n, a in W.generate(wl, wq_gain=g, heads=1).items() if n not in ("q", "k", "v")})
+        den_l = O.phi_features(q[rows], head_weights(dg, "q", 0), wl.degree) @ z
         return float(np.median(lam * den_l / den_s))
 
     lo, hi = 1e-6, 1.0
     if ratio(hi) <= 1.0:
         return 1.0
-    for _ in range(60):
+    for _ in range(40):
         mid = math.sqrt(lo * hi)
         if ratio(mid) > 1.0:
             hi = mid
@@ -178,8 +189,17 @@ def oracle_eval(wl, data64, stab_mode, rows=None, key=None):
     inputs is compared with the same oracle output without evaluating it again."""
     if key is not None and key in _ORACLE_CACHE:
         return _ORACLE_CACHE[key]
-    res = O.hybrid_attention(data64["q"], data64["k"], data64["v"], data64["wq"], data64["wk"],
-                             oracle_mask(wl), None, stab_mode, wl.degree, rows=rows)
+    mask = oracle_mask(wl)
+    B, H, N, d = data64["q"].shape
+    n_rows = N if rows is None else len(rows)
+    y = np.empty((B, H, n_rows, d))
+    aux = np.empty((B, H, n_rows, 3))
+    for b in range(B):
+        for h in range(H):
+            y[b, h], aux[b, h] = O.hybrid_attention_head(
+                data64["q"][b, h], data64["k"][b, h], data64["v"][b, h], head_weights(data64, "q", h),
+                head_weights(data64, "k", h), mask, None, stab_mode, wl.degree, rows=rows)
+    res = (y, aux)
     if key is not None:
         _ORACLE_CACHE.clear()
         _ORACLE_CACHE[key] = res
@@ -194,5 +214,5 @@ def oracle_state(wl, data64):
     z = np.empty((B, H, wl.F))
     for b in range(B):
         for h in range(H):
-            S[b, h], z[b, h] = O.linear_state(data64["k"][b, h], data64["v"][b, h], data64["wk"][h], mask, wl.degree)
+            S[b, h], z[b, h] = O.linear_state(data64["k"][b, h], data64["v"][b, h], head_weights(data64, "k", h), mask, wl.degree)
     return S, z

@@ -62,8 +62,14 @@ def _desc(**kw):
     (dict(softmax_idx=[5, 2000]), binding.AS_ERR_INVALID_ARG),   # out of range
     (dict(poly_degree=3), binding.AS_ERR_INVALID_ARG),           # 64 not divisible by 3
     (dict(d=96, phi_dim=96), binding.AS_ERR_UNSUPPORTED),
-    (dict(phi_dim=128), binding.AS_ERR_UNSUPPORTED),             # F != d has no kernel yet
-    (dict(phi_layers=2, phi_hidden=128), binding.AS_ERR_UNSUPPORTED),
+    (dict(phi_dim=192), binding.AS_ERR_UNSUPPORTED),             # neither d nor a multiple of 128
+    (dict(phi_dim=640), binding.AS_ERR_UNSUPPORTED),             # more than 512 features
+    (dict(poly_degree=4), binding.AS_ERR_UNSUPPORTED),           # parts of 16 features: not a multiple of 32
+    (dict(phi_layers=2, phi_hidden=128), binding.AS_ERR_UNSUPPORTED),   # at d = 64 two layers need hidden = F = d
+    (dict(d=128, phi_dim=256, phi_layers=2, phi_hidden=512), binding.AS_ERR_UNSUPPORTED),
+    (dict(d=128, phi_dim=384, phi_layers=2, phi_hidden=128), binding.AS_ERR_UNSUPPORTED),
+    (dict(phi_layers=3, phi_hidden=64), binding.AS_ERR_UNSUPPORTED),
+    (dict(phi_dim=128, kernel_path=binding.AS_PATH_SIMT), binding.AS_ERR_UNSUPPORTED),   # the check path has F = d only
 ])
 def test_create_rejects_bad_descriptors(lib, kw, status):
     h = C.c_void_p()

@@ -58,7 +58,8 @@ def _run(wl, path, mode, gain=1.0, rows=None, heads=None, want_state=False, soft
     out = g_out.view(torch.bfloat16, (wl.B, wl.H, wl.N, wl.d))
     aux = g_aux.view(torch.float32, (wl.B, wl.H, wl.N, 3))
     aux.fill_(float("nan"))
-    op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], out=out, aux=aux, workspace=g_ws.bytes())
+    op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], out=out, aux=aux, workspace=g_ws.bytes(),
+               wq2=dev.get("wq2"), wk2=dev.get("wk2"), biases={n: t for n, t in dev.items() if n.startswith("b")} or None)
     torch.cuda.synchronize()
     assert op.last_status() == 0
     for g, name in ((g_out, "out"), (g_aux, "aux"), (g_ws, "workspace")):
@@ -346,6 +347,32 @@ def test_run_to_run_determinism_and_launch_count():
     assert cnt == [1, 1, 1] and all(t > 0 for t in ms)
 
 
+def test_expired_device_wait_is_reported_once_and_the_handle_recovers():
+    """The time-out path in its safe form: a dedicated kernel's bounded wait runs out (nothing else is in flight),
+    the status word is set, forwards on the handle do nothing until the word has been read, last_status reports
+    the time-out once, and the next forward is correct again."""
+    import torch
+    from paper_2509_24899_b200 import HybridAttention, binding
+    wl = SMALL["one_tile"]
+    data = W.generate(wl, wq_gain=0.02)
+    dev = {k: to_cuda_bf16(v) for k, v in data.items()}
+    op = HybridAttention.from_workload(wl)
+    good = op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"]).clone()
+    torch.cuda.synchronize()
+    assert op.last_status() == 0
+    st = torch.cuda.current_stream().cuda_stream
+    binding.as_hybrid_attn_debug_expire_wait(op.handle, 2_000_000, st)       # about a millisecond
+    sentinel = torch.full_like(good, 7.0)
+    op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], out=sentinel)   # inert: kernels return at once
+    torch.cuda.synchronize()
+    assert torch.equal(sentinel, torch.full_like(good, 7.0))
+    assert op.last_status() == binding.AS_ERR_DEVICE_TIMEOUT
+    assert op.last_status() == 0                                               # read and cleared
+    again = op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"])
+    torch.cuda.synchronize()
+    assert op.last_status() == 0 and torch.equal(again, good)
+
+
 def test_gpu_argument_errors():
     import torch
     from paper_2509_24899_b200 import HybridAttention, binding, AsError
@@ -379,58 +406,67 @@ TWO_LAYER = {
                                   rate=0, seed=33, layers=2),
     "two_layer_chunks": W.Workload("two_layer_chunks", B=1, H=1, d=128, F=128, grid=(8, 30, 52), block=(1, 6, 8),
                                    rate=8, seed=34, layers=2),
-    # more (batch, head) pairs than SMs: several units per persistent CTA, with the two first-layer tiles,
-    # the weights and the last V tile competing for the three ring slots at every unit's end
+    # more (batch, head) pairs than SMs: several units per persistent CTA, with the weight tiles of the tail and the
+    # last V tile competing for the three ring slots at every unit's end
     "two_layer_many_units": W.Workload("two_layer_many_units", B=2, H=80, d=128, F=128, grid=(1, 10, 30), block=(1, 5, 6),
                                        rate=3, seed=35, layers=2),
     "two_layer_many_units_rate0": W.Workload("two_layer_many_units_rate0", B=2, H=80, d=64, F=64, grid=(1, 10, 30),
                                              block=(1, 5, 6), rate=0, seed=36, layers=2, rms_norm_qk=False),
 }
 
-
-def _oracle_two_layer(wl, d64, mode, rows=None):
-    """Oracle with the two-layer embedding network: the weights of a head are the list [W_1, W_2]."""
-    mask = oracle_mask(wl)
-    B, H = d64["q"].shape[:2]
-    n_rows = wl.N if rows is None else len(rows)
-    y = np.empty((B, H, n_rows, wl.d))
-    aux = np.empty((B, H, n_rows, 3))
-    S = np.empty((B, H, wl.F, wl.d))
-    z = np.empty((B, H, wl.F))
-    for b in range(B):
-        for h in range(H):
-            wq, wk = [d64["wq"][h], d64["wq2"][h]], [d64["wk"][h], d64["wk2"][h]]
-            y[b, h], aux[b, h] = O.hybrid_attention_head(d64["q"][b, h], d64["k"][b, h], d64["v"][b, h], wq, wk, mask,
-                                                         None, mode, wl.degree, rows=rows)
-            if not mask.all():
-                S[b, h], z[b, h] = O.linear_state(d64["k"][b, h], d64["v"][b, h], wk, mask, wl.degree)
-    return y, aux, S, z
+# Feature maps wider than the head ("Characterization of phi": d -> P*d -> P*d, Table of phi sizes), polynomial
+# degrees up to 4, biases.  paper_default is the paper's default map: two layers, hidden = F = 2d, degree 2.
+WIDE = {
+    "f256_one_layer": W.Workload("f256_one_layer", B=1, H=2, d=128, F=256, grid=(3, 10, 13), block=(1, 6, 8), rate=4, seed=41),
+    "f384_degree3": W.Workload("f384_degree3", B=1, H=2, d=128, F=384, grid=(3, 10, 13), block=(1, 6, 8), rate=4, seed=42, degree=3),
+    "f512_degree4_bias": W.Workload("f512_degree4_bias", B=1, H=2, d=128, F=512, grid=(3, 10, 13), block=(1, 6, 8), rate=3,
+                                    seed=43, degree=4, bias=True),
+    "f128_degree4": W.Workload("f128_degree4", B=1, H=2, d=128, F=128, grid=(3, 10, 13), block=(1, 6, 8), rate=4, seed=44, degree=4),
+    "f128_bias": W.Workload("f128_bias", B=1, H=2, d=128, F=128, grid=(3, 10, 13), block=(1, 6, 8), rate=4, seed=45, bias=True),
+    "d64_f128": W.Workload("d64_f128", B=2, H=3, d=64, F=128, grid=(2, 9, 31), block=(1, 4, 4), rate=2, seed=46, rms_norm_qk=False),
+    "d64_f256_bias": W.Workload("d64_f256_bias", B=1, H=2, d=64, F=256, grid=(2, 9, 31), block=(1, 4, 4), rate=2, seed=47,
+                                rms_norm_qk=False, bias=True),
+    "f256_rate0": W.Workload("f256_rate0", B=1, H=2, d=128, F=256, grid=(3, 10, 13), block=(1, 6, 8), rate=0, seed=48),
+    "f256_many_units": W.Workload("f256_many_units", B=2, H=80, d=128, F=256, grid=(1, 10, 30), block=(1, 5, 6), rate=3, seed=49),
+    "f256_chunks": W.Workload("f256_chunks", B=1, H=1, d=128, F=256, grid=(8, 30, 52), block=(1, 6, 8), rate=8, seed=50),
+    "paper_default": W.Workload("paper_default", B=1, H=2, d=128, F=256, grid=(3, 10, 13), block=(1, 6, 8), rate=4, seed=51,
+                                layers=2, hidden=256),
+    "paper_default_bias": W.Workload("paper_default_bias", B=1, H=2, d=128, F=256, grid=(3, 10, 13), block=(1, 6, 8), rate=4,
+                                     seed=52, layers=2, hidden=256, bias=True),
+    "paper_default_rate0": W.Workload("paper_default_rate0", B=1, H=2, d=128, F=256, grid=(3, 10, 13), block=(1, 6, 8), rate=0,
+                                      seed=53, layers=2, hidden=256),
+    "paper_default_many_units": W.Workload("paper_default_many_units", B=2, H=80, d=128, F=256, grid=(1, 10, 30), block=(1, 5, 6),
+                                           rate=3, seed=54, layers=2, hidden=256),
+    "paper_default_chunks": W.Workload("paper_default_chunks", B=1, H=1, d=128, F=256, grid=(8, 30, 52), block=(1, 6, 8), rate=8,
+                                       seed=55, layers=2, hidden=256),
+    "hidden256_f128": W.Workload("hidden256_f128", B=1, H=2, d=128, F=128, grid=(3, 10, 13), block=(1, 6, 8), rate=4, seed=56,
+                                 layers=2, hidden=256),
+    "hidden128_f256_bias": W.Workload("hidden128_f256_bias", B=1, H=2, d=128, F=256, grid=(3, 10, 13), block=(1, 6, 8), rate=4,
+                                      seed=57, layers=2, hidden=128, bias=True),
+    "two_layer_d64_bias": W.Workload("two_layer_d64_bias", B=2, H=3, d=64, F=64, grid=(2, 9, 31), block=(1, 4, 4), rate=2, seed=58,
+                                     rms_norm_qk=False, layers=2, bias=True),
+}
+FEATURE_MAPS = dict(TWO_LAYER, **WIDE)
 
 
 @pytest.mark.parametrize("mode", MODES)
-@pytest.mark.parametrize("name", sorted(TWO_LAYER))
-def test_two_layer_feature_map(mode, name):
-    """phi(x) = poly(ReLU(W_2 ReLU(W_1 x))): first layer by its own kernel, second layer fused into the K and Q pass."""
-    import torch
-    from paper_2509_24899_b200 import HybridAttention
-    wl = TWO_LAYER[name]
-    data = W.generate(wl, wq_gain=0.05 if wl.rate else 1.0)
-    dev = {k: to_cuda_bf16(v) for k, v in data.items()}
-    op = HybridAttention.from_workload(wl, stab_mode=mode)
-    aux = torch.full((wl.B, wl.H, wl.N, 3), float("nan"), dtype=torch.float32, device="cuda")
-    out = op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], aux=aux, wq2=dev["wq2"], wk2=dev["wk2"])
-    Sg, zg = op.linear_state()
-    torch.cuda.synchronize()
-    assert op.last_status() == 0
-    d64 = oracle_inputs(data)
-    ref, ref_aux, S, z = _oracle_two_layer(wl, d64, mode)
-    assert errors(Sg.cpu().numpy().astype(np.float64), S)[0] <= 5e-3
-    assert errors(zg.cpu().numpy().astype(np.float64), z)[0] <= 5e-3
-    got = from_cuda_bf16(out)
+@pytest.mark.parametrize("name", sorted(FEATURE_MAPS))
+def test_feature_map_shapes(mode, name):
+    """Deeper and wider feature maps: two layers (first layer of the keys by its own kernel, of the queries inside the
+    Q pass), up to 512 features in chunks of 128, polynomial degrees up to 4, biases."""
+    wl = FEATURE_MAPS[name]
+    gain = balanced_gain(wl, mode)
+    got, got_aux, ref, ref_aux, ex = _run(wl, FULL_PATH, mode, gain, want_state=True)
+    S, z = oracle_state(wl, ex["data64"])
+    assert errors(ex["S"], S)[0] <= 5e-3 and errors(ex["z"], z)[0] <= 5e-3
     ok = np.isfinite(ref).all(-1)
     assert ok.mean() > 0.99
-    assert_parity(got[ok], ref[ok], _tag(name, "tensor", mode))
-    _check_aux(aux.cpu().numpy().astype(np.float64)[ok], ref_aux[ok], wl, op.n_softmax)
+    assert_parity(got[ok], ref[ok], _tag(name, FULL_PATH, mode, True))
+    _check_aux(got_aux[ok], ref_aux[ok], wl, ex["n_softmax"])
+    if wl.rate not in (0, 1):
+        lam = np.exp(-ref_aux[..., 0]) if mode == O.STAB_EXACT else 1.0
+        ratio = np.median((lam * ref_aux[..., 2] / ref_aux[..., 1])[ok])
+        assert 0.2 < ratio < 5.0          # both branches carry weight
 
 
 def test_two_layer_needs_its_second_weights_and_the_tensor_path():
@@ -443,6 +479,10 @@ def test_two_layer_needs_its_second_weights_and_the_tensor_path():
     dev = {k: to_cuda_bf16(v) for k, v in W.generate(wl).items()}
     with pytest.raises(AsError) as e:
         op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"])
+    assert e.value.status == binding.AS_ERR_INVALID_ARG
+    with pytest.raises(AsError) as e:          # a bias that is not 4-byte aligned
+        op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], wq2=dev["wq2"], wk2=dev["wk2"],
+                   biases={"bq1": dev["wq"].view(-1)[1:]})
     assert e.value.status == binding.AS_ERR_INVALID_ARG
 
 
