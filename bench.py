@@ -26,9 +26,38 @@ sys.path.insert(0, ROOT)
 
 METRIC = "hybrid-attn fwd tokens/s per layer at N=32760 (12x128 heads); % of bf16 tensor peak"
 
-# DRAM bytes of one Q-pass launch at the wan81 workload (dram__bytes_read.sum + dram__bytes_write.sum
-# from the ncu capture summarised in profiles/); None until a capture exists.
-QPASS_DRAM_TRAFFIC_BYTES = {"wan81": 126750464 + 63403008}
+KERNEL_SOURCES = ("tensor_qpass.cu", "tensor_common.cuh", "sm100_ptx.cuh", "sm100_tmem_wide.cuh")
+
+
+def kernel_source_digest(names=KERNEL_SOURCES):
+    """sha256 over the source files a kernel is built from (the ncu summaries record it at capture time)."""
+    import hashlib
+    h = hashlib.sha256()
+    for n in names:
+        with open(os.path.join(ROOT, "paper_2509_24899_b200", "csrc", n), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def measured_dram_traffic(kernel, workload):
+    """DRAM bytes of one launch (dram__bytes_read.sum + dram__bytes_write.sum) from the committed ncu summary
+    profiles/<kernel>_<workload>.txt, or None when there is no summary or the kernel's sources have changed
+    since the capture (the summary carries the digest of the sources it was taken with)."""
+    path = os.path.join(ROOT, "profiles", "%s_%s.txt" % (kernel, workload))
+    if not os.path.exists(path):
+        return None
+    fields = {}
+    with open(path) as f:
+        for line in f:
+            if ":" in line:
+                k, v = line.split(":", 1)
+                fields[k.strip()] = v.strip()
+    try:
+        if fields["source_digest"] != kernel_source_digest():
+            return None
+        return int(fields["dram_bytes_read_per_launch"]) + int(fields["dram_bytes_write_per_launch"])
+    except (KeyError, ValueError):
+        return None
 
 
 def _peaks():
@@ -42,18 +71,28 @@ def _peaks():
 
 
 def flops_per_layer(wl, n_s):
-    """Algorithmic FLOPs of one layer (all heads), split per kernel."""
+    """Algorithmic FLOPs of one layer (all heads), split per kernel.  Per token the feature map costs
+    2 d F (one layer) or 2 d hidden + 2 hidden F (two layers); state and apply cost 2 F (d + 1) each."""
     N, d, F = wl.N, wl.d, wl.F
     n_l = N - n_s
     heads = wl.B * wl.H
-    kpass = (2 * d * F * n_l + 2 * n_l * F * (d + 1)) if n_l > 0 else 0
-    qpass = 4 * N * n_s * d + ((2 * N * d * F + 2 * N * F * (d + 1)) if n_l > 0 else 0)
+    phi = 2 * d * F if wl.layers == 1 else 2 * d * wl.hidden_width + 2 * wl.hidden_width * F
+    kpass = (phi * n_l + 2 * n_l * F * (d + 1)) if n_l > 0 else 0
+    qpass = 4 * N * n_s * d + ((N * phi + 2 * N * F * (d + 1)) if n_l > 0 else 0)
     return {"kpass": heads * kpass, "qpass": heads * qpass, "total": heads * (kpass + qpass)}
 
 
 def bytes_per_layer(wl):
     """Algorithmic HBM bytes of one layer: q, k, v read once, out written once."""
     return 4 * wl.B * wl.H * wl.N * wl.d * 2
+
+
+def config_of(wl, n_softmax, world):
+    """The `config` object of the JSON line: the workload, named the same way by both arms."""
+    return {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "d": wl.d, "F": wl.F, "rate": wl.rate,
+            "n_softmax": int(n_softmax), "stab_mode": "paper",
+            "phi": "%d layer(s), hidden %d, F %d, degree %d" % (wl.layers, wl.hidden_width if wl.layers == 2 else 0, wl.F, wl.degree),
+            "parallelism": "dp%d (independent layer inputs per rank)" % world}
 
 
 def rank_workload(wl, rank):
@@ -119,6 +158,9 @@ class ClockSampler:
         if self.ok:
             self.thread.start()
 
+    def reset(self):
+        self.samples = []
+
     def stop(self):
         self._stop.set()
         if self.ok and self.thread.is_alive():
@@ -138,6 +180,17 @@ class ClockSampler:
                 "reasons": sorted(seen), "samples": len(self.samples)}
 
 
+def head_weights(data64, which, h):
+    """One head's feature map in the form the oracle takes: a matrix, or a list of layers, each a matrix or a
+    (matrix, bias) pair (argument marshalling only)."""
+    def layer(wname, bname):
+        return (data64[wname][h], data64[bname][h]) if bname in data64 else data64[wname][h]
+    first = layer("w" + which, "b" + which + "1")
+    if ("w" + which + "2") not in data64:
+        return first if not isinstance(first, tuple) else [first]
+    return [first, layer("w" + which + "2", "b" + which + "2")]
+
+
 def cpu_oracle_rate(wl, data64, mask, budget_s, heads=1, rows0=256):
     """Times the float64 oracle on a bounded sample and extrapolates to tokens/s of a full layer.
 
@@ -154,11 +207,11 @@ def cpu_oracle_rate(wl, data64, mask, budget_s, heads=1, rows0=256):
         for h in range(heads):
             if n_l > 0:
                 t0 = time.perf_counter()
-                O.linear_state(k[h], v[h], data64["wk"][h], mask, wl.degree)
+                O.linear_state(k[h], v[h], head_weights(data64, "k", h), mask, wl.degree)
                 t_state += time.perf_counter() - t0
             t0 = time.perf_counter()
-            O.hybrid_attention_head(q[h], k[h], v[h], data64["wq"][h], data64["wk"][h], mask, None,
-                                    O.STAB_PAPER, wl.degree, rows=rows)
+            O.hybrid_attention_head(q[h], k[h], v[h], head_weights(data64, "q", h), head_weights(data64, "k", h), mask,
+                                    None, O.STAB_PAPER, wl.degree, rows=rows)
             t_rows += time.perf_counter() - t0
         return t_state / heads, t_rows / heads
 
@@ -201,8 +254,7 @@ def run_reference(args, wl):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wl.B * wl.N / value,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "d": wl.d, "F": wl.F,
-                   "rate": wl.rate, "n_softmax": int(mask.sum())},
+        "config": config_of(wl, mask.sum(), args.gpus),
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
                          "sample": "per step: 1 head, linear state over all tokens + %d query rows against all "
                                    "keys; extrapolated to H heads x N rows" % last["rows"]},
@@ -239,13 +291,25 @@ def run_ours(args, wl):
     data = W.generate(wl_r)
     to_dev = lambda b: torch.from_numpy(b.view(np.int16)).cuda().view(torch.bfloat16)
     dev = {k: to_dev(v) for k, v in data.items()}
+    weights = {k: v for k, v in dev.items() if k not in ("q", "k", "v")}
+    # The step's inputs rotate over several copies in HBM (distinct addresses), so that no step finds its q, k, v
+    # in L2 from the step before; three sets of inputs plus the output exceed the 126 MB L2 many times over.
+    n_sets = 1 if args.skip_extras else max(1, min(3, int(6e9 // (3 * dev["q"].numel() * 2))))
+    sets = [{k: dev[k] for k in ("q", "k", "v")}] + [{k: dev[k].clone() for k in ("q", "k", "v")} for _ in range(n_sets - 1)]
     path = {"tensor": binding.AS_PATH_TENSOR, "simt": binding.AS_PATH_SIMT}[args.path]
     op = HybridAttention.from_workload(wl_r, kernel_path=path)
     out = torch.empty_like(dev["q"])
     stream = torch.cuda.current_stream()
-    step = lambda: op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], out=out, stream=stream)
+    fw = dict(wq2=weights.get("wq2"), wk2=weights.get("wk2"),
+              biases={n: t for n, t in weights.items() if n.startswith("b")} or None)
+    counter = [0]
 
-    sampler = ClockSampler(local)
+    def step():
+        x = sets[counter[0] % n_sets]
+        counter[0] += 1
+        op.forward(x["q"], x["k"], x["v"], weights["wq"], weights["wk"], out=out, stream=stream, **fw)
+
+    sampler = ClockSampler(local, period_s=0.005)
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
@@ -256,6 +320,7 @@ def run_ours(args, wl):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler.start()
     barrier()
+    sampler.reset()
     e0.record(stream)
     for _ in range(args.steps):
         step()
@@ -266,6 +331,26 @@ def run_ours(args, wl):
     kms, kcnt = binding.as_hybrid_attn_profile_read(op.handle)
     binding.as_hybrid_attn_profile_enable(op.handle, False)
     status = op.last_status()
+    burst_clocks = sampler.summary()
+
+    # A second, longer region (about two seconds): the same step under the power cap, with the SM clock sampled
+    # inside it, so that the line carries a burst and a sustained figure side by side.
+    sustained = None
+    if not args.skip_extras and args.sustained_s > 0:
+        n_sus = max(args.steps, int(args.sustained_s * 1e3 / max(ms / args.steps, 1e-3)))
+        sampler.reset()
+        barrier()
+        e0.record(stream)
+        for _ in range(n_sus):
+            step()
+        e1.record(stream)
+        barrier()
+        sus_ms = e0.elapsed_time(e1)
+        sus_clocks = sampler.summary()
+        (sus_ms,) = max_over_ranks([sus_ms], "cuda")
+        sustained = {"steps": n_sus, "seconds": sus_ms * 1e-3, "ms_per_step": sus_ms / n_sus,
+                     "value": whole_job_value(wl, world, n_sus, sus_ms), "clocks": sus_clocks}
+        status = status or op.last_status()
 
     if args.skip_extras:          # profiling runs: only the device-timed region
         if rank == 0:
@@ -280,11 +365,11 @@ def run_ours(args, wl):
     out_host = torch.empty_like(host["q"]).pin_memory()
     e2e_steps = max(3, min(args.steps, 20))
     for _ in range(2):
-        op.forward_host(host["q"], host["k"], host["v"], dev["wq"], dev["wk"], out_host, stream=stream)
+        op.forward_host(host["q"], host["k"], host["v"], weights["wq"], weights["wk"], out_host, stream=stream, **fw)
     barrier()
     e0.record(stream)
     for _ in range(e2e_steps):
-        op.forward_host(host["q"], host["k"], host["v"], dev["wq"], dev["wk"], out_host, stream=stream)
+        op.forward_host(host["q"], host["k"], host["v"], weights["wq"], weights["wk"], out_host, stream=stream, **fw)
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1)
@@ -307,11 +392,12 @@ def run_ours(args, wl):
             achieved = fl["qpass"] / (q_ms * 1e-3) / 1e12
             roof = {"bound": "tensor", "kernel": "qpass", "achieved": achieved, "peak": peaks["bf16_tflops"],
                     "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
-                    "traffic": QPASS_DRAM_TRAFFIC_BYTES.get(wl.name),
+                    "traffic": measured_dram_traffic("qpass_kernel", wl.name),
                     "peak_source": "%s burst bf16 (sustained %s)" % (peaks["source"], peaks["bf16_tflops_sustained"]),
                     "frac_of_nominal_2250": achieved / 2250.0,
                     "frac_of_sustained": (achieved / peaks["bf16_tflops_sustained"]) if peaks.get("bf16_tflops_sustained") else None,
                     "avg_launch_ms": q_ms,
+                    "avg_launch_sm_cycles": (q_ms * 1e-3 * burst_clocks["sm_mhz"] * 1e6) if burst_clocks.get("sm_mhz") else None,
                     "flops_per_launch": fl["qpass"]}
         else:       # rate 0: the whole layer is bound by reading q, k, v and writing out
             gbs = bytes_per_layer(wl) / ((k_ms + r_ms + q_ms) * 1e-3) / 1e9
@@ -324,15 +410,21 @@ def run_ours(args, wl):
         d1 = {k: W.bf16_bits_to_f64(v[:, :1] if k in ("q", "k", "v") else v[:1]) for k, v in data.items()}
         mask = O.softmax_token_mask(wl.grid, wl.block, wl.rate)
         cb = cpu_oracle_rate(wl, d1, mask, budget_s=15.0, heads=1)
-        clocks = sampler.summary()
+        clocks = burst_clocks if burst_clocks.get("samples", 0) >= 2 or sustained is None else sustained["clocks"]
+        if sustained is not None:
+            sus_tflops = fl["total"] / (sustained["ms_per_step"] * 1e-3) / 1e12
+            sustained.update({"tflops": sus_tflops, "frac_of_nominal_2250": sus_tflops / 2250.0,
+                              "peak": peaks.get("bf16_tflops_sustained"),
+                              "frac_of_sustained_peak": (sus_tflops / peaks["bf16_tflops_sustained"])
+                              if peaks.get("bf16_tflops_sustained") else None})
         line = {
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "d": wl.d, "F": wl.F,
-                       "rate": wl.rate, "n_softmax": n_s, "stab_mode": "paper", "kernel_path": args.path,
-                       "l2": "q,k,v,out of a step total %.0f MB > 126 MB L2" % (bytes_per_layer(wl) / 1e6),
-                       "parallelism": "dp%d (independent layer inputs per rank)" % world},
+            "config": config_of(wl, n_s, world),
+            "timing": {"kernel_path": args.path,
+                       "l2": "q,k,v,out of a step total %.0f MB > 126 MB L2; inputs rotate over %d sets of buffers"
+                             % (bytes_per_layer(wl) / 1e6, n_sets)},
             "tflops": fl["total"] * args.steps / (ms * 1e-3) / 1e12 * 1.0,
             "kernel_ms": {"kpass": k_ms, "reduce": r_ms, "qpass": q_ms},
             "roofline": roof,
@@ -343,6 +435,7 @@ def run_ours(args, wl):
                     "h2d_bytes_per_step": 3 * wl.B * wl.H * wl.N * wl.d * 2,
                     "d2h_bytes_per_step": wl.B * wl.H * wl.N * wl.d * 2, "steps": e2e_steps},
             "gpu_launches": int(launches),
+            "sustained": sustained,
             "clocks": clocks,
             "device_status": status,
         }
@@ -410,9 +503,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="wan81",
-                    help="tiny | wan17 | wan81 | wan161cfg | stack:<layer> | stack (all five rates, summed)")
+                    help="tiny | wan17 | wan81 | wan161cfg | stack:<layer> | stack (all five rates, summed) | "
+                         "wan81_paper_phi | wan81_f256 (the headline layer with wider feature maps)")
     ap.add_argument("--path", default="tensor", choices=["tensor", "simt"],
                     help="kernel path: tcgen05 tensor-core kernels (default) or the fp32 CUDA-core check path")
+    ap.add_argument("--sustained-s", type=float, default=2.0,
+                    help="length in seconds of the second, power-capped timed region (0 = none)")
     ap.add_argument("--skip-extras", action="store_true",
                     help="only the device-timed steps (for profiler runs): no e2e, no CPU baseline")
     args = ap.parse_args()
@@ -421,6 +517,8 @@ def main():
         return run_stack(args)
     if args.workload.startswith("stack:"):
         wl = W.stack_layer(int(args.workload.split(":")[1]))
+    elif args.workload in W.VARIANTS:
+        wl = W.VARIANTS[args.workload]
     else:
         wl = W.CONFIGS[args.workload]
     if args.impl == "reference":

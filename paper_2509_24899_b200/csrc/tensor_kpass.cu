@@ -47,6 +47,10 @@ struct KLayout {
   static constexpr int PAIR_OFF = BAR_OFF + 8 * N_BARS + 16;    // 2 x 64 words: per token pair, which halves are linear tokens
   static constexpr int Z_OFF = PAIR_OFF + 2 * 64 * 4;           // 128 floats: z of the upper column half
   static constexpr int TOTAL = Z_OFF + 128 * 4 + 1024;          // + slack for the 1024-byte alignment
+  // the chunk's partial S leaves through the ring (idle by then): 128 rows of D floats, each row padded by 16
+  // bytes so that the 32 lanes of a warp, one row each, write to different banks
+  static constexpr int OUT_PITCH = D * 4 + 16;
+  static_assert(128 * OUT_PITCH <= SLOTS * TILE, "staging area");
 };
 
 // Features of 32 token columns of one TMEM lane: bias, ReLU, power, linear-token mask, bf16.
@@ -102,16 +106,38 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   __syncthreads();
   if (s_skip != 0u) return;
 
+  auto sW = [&](int j) { return sbase + L::W_OFF + j * L::TILE; };
+  auto sSlot = [&](int it) { return sbase + L::RING_OFF + (it % SLOTS) * L::TILE; };
+  // one ring item: tile t's K (one layer) or hidden slice i (two layers), or its V tile
+  auto load_item = [&](int it) {
+    const int st = it % SLOTS, t = it / IPT, i = it % IPT, row = (t_begin + t) * 128;
+    mbar_expect_tx(bar(B_FULL + st), L::TILE);
+    if (i == NX) load_tile<D>(sSlot(it), &tmV, bar(B_FULL + st), row, bh);
+    else if (LAYERS == 1) load_tile<D>(sSlot(it), &tmK, bar(B_FULL + st), row, bh);
+    else load_boxes(sSlot(it), &tmH, bar(B_FULL + st), i * D, row, bh, D / 64);
+  };
+  constexpr int FIRST = SLOTS;                               // items requested before the CTA has finished setting up: the whole ring
+
   if (threadIdx.x == 0) {
     *abort_flag = 0u;
+    for (int b = 0; b < 2; ++b) { mbar_init(bar(B_D1 + b), 1); mbar_init(bar(B_PK + b), K_FEATURE_THREADS); }
+    mbar_init(bar(B_DONE), 1);
+    fence_barrier_init();
+  }
+  if (threadIdx.x == 8 * 32) {
+    // The producer sets up the barriers of the ring itself and requests the weights and the first tiles at
+    // once: the first bytes of a CTA take several microseconds to arrive, and the allocation of tensor memory
+    // and the CTA-wide barrier below need not be waited for.
     mbar_init(bar(B_W), 1);
     // a slot is free again when the MMA that read it has completed and, where rows are gathered, when both
     // gather warps are through with it
     for (int s = 0; s < SLOTS; ++s) { mbar_init(bar(B_FULL + s), 1); mbar_init(bar(B_EMPTY + s), gathers ? 3 : 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(bar(B_D1 + b), 1); mbar_init(bar(B_PK + b), K_FEATURE_THREADS); }
-    mbar_init(bar(B_DONE), 1);
     fence_barrier_init();
     fence_proxy_async();
+    mbar_expect_tx(bar(B_W), NH * L::TILE);
+    // rows past F are out of bounds and arrive as zeros
+    for (int j = 0; j < NH; ++j) load_boxes(sW(j), &tmW, bar(B_W), j * D, fc * 128, h, D / 64);
+    for (int it = 0; it < FIRST && it < nt * IPT; ++it) load_item(it);
   }
   if (warp == 9) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
   tc_fence_before();
@@ -121,60 +147,73 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   const uint32_t tD1[2] = {tmem + 0u, tmem + 128u};          // Phi^T of a tile, fp32
   const uint32_t tAcc = tmem + 256u;                         // S of this feature chunk
   const uint32_t tPA[2] = {tmem + 384u, tmem + 448u};        // the tile's features as packed bf16 (A operand)
-  auto sW = [&](int j) { return sbase + L::W_OFF + j * L::TILE; };
-  auto sSlot = [&](int it) { return sbase + L::RING_OFF + (it % SLOTS) * L::TILE; };
 
   if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmW); tma_prefetch_desc(&tmH);
-      mbar_expect_tx(bar(B_W), NH * L::TILE);
-      // rows past F are out of bounds and arrive as zeros
-      for (int j = 0; j < NH; ++j) load_boxes(sW(j), &tmW, bar(B_W), j * D, fc * 128, h, D / 64);
-    }
-    for (int it = 0; it < nt * IPT; ++it) {
+    for (int it = FIRST; it < nt * IPT; ++it) {              // the first items were requested during set-up
       const int st = it % SLOTS;
       if (!mbar_wait_warp(bar(B_EMPTY + st), ((it / SLOTS) & 1) ^ 1, wc)) break;
-      if (lane == 0) {
-        const int t = it / IPT, i = it % IPT, row = (t_begin + t) * 128;
-        mbar_expect_tx(bar(B_FULL + st), L::TILE);
-        if (i == NX) load_tile<D>(sSlot(it), &tmV, bar(B_FULL + st), row, bh);
-        else if (LAYERS == 1) load_tile<D>(sSlot(it), &tmK, bar(B_FULL + st), row, bh);
-        else load_boxes(sSlot(it), &tmH, bar(B_FULL + st), i * D, row, bh, D / 64);
-      }
+      if (lane == 0) load_item(it);
       __syncwarp();
     }
   } else if (warp == 9) {
     // ------------------------------------------------------------ MMA issuer (one thread)
+    // Two kinds of product per tile: Phi^T(t) as soon as the tile's X items have landed, and S += phi^T V (t) as
+    // soon as the feature warps have packed the tile.  The thread issues whichever is ready, so that neither a
+    // late tile holds up the accumulation of an earlier one (and with it the release of its V slot) nor the
+    // other way round.  Phi^T(t) reuses the columns the feature warps read for tile t - 2 and its features will
+    // overwrite the packed operand of S(t - 2): it is only issued once S(t - 2) has been (products of one thread
+    // complete in order).
     if (lane == 0) {
       constexpr uint32_t ID_PHI = make_idesc(128, 128, 0, 0);    // Phi^T = W X^T : M = features, N = 128 tokens
       constexpr uint32_t ID_ACC = make_idesc(128, D, 0, 1);      // S += phi^T V  : V is MN-major
       bool ok = mbar_wait(bar(B_W), 0, wc);
-      for (int t = 0; ok && t <= nt; ++t) {
-        if (t < nt) {
-#pragma unroll
-          for (int j = 0; j < NX; ++j) {
-            const int it = t * IPT + j;
-            ok = ok && mbar_wait(bar(B_FULL + it % SLOTS), (it / SLOTS) & 1, wc);
-          }
-          if (!ok) break;
-          tc_fence_after();
-#pragma unroll
-          for (int j = 0; j < NX; ++j) {
-            const int it = t * IPT + j;
-            issue_kmajor<D>(tD1[t & 1], kmajor_desc(sW(j)), kmajor_desc(sSlot(it)), ID_PHI, j > 0);
+      int tp = 0, ts = 0;                                        // next tile for Phi^T / for the accumulation
+      long long t0 = 0;
+      uint32_t polls = 0;
+      while (ok && ts < nt) {
+        bool did = false;
+        if (ts < tp) {                                           // S(ts): packed features and the V tile
+          const int it = ts * IPT + NX;
+          if (mbar_try_wait(bar(B_PK + (ts & 1)), (ts >> 1) & 1) && mbar_try_wait(bar(B_FULL + it % SLOTS), (it / SLOTS) & 1)) {
+            tc_fence_after();
+            issue_tmemA_mnB(tAcc, tPA[ts & 1], mnmajor_desc(sSlot(it)), ID_ACC, ts > 0);
             tc_commit(bar(B_EMPTY + it % SLOTS));
+            if (ts == nt - 1) tc_commit(bar(B_DONE));
+            ++ts;
+            did = true;
           }
-          tc_commit(bar(B_D1 + (t & 1)));
         }
-        if (t >= 1) {
-          const int u = t - 1, it = u * IPT + NX;
-          ok = mbar_wait(bar(B_PK + (u & 1)), (u >> 1) & 1, wc) && mbar_wait(bar(B_FULL + it % SLOTS), (it / SLOTS) & 1, wc);
-          if (!ok) break;
-          tc_fence_after();
-          issue_tmemA_mnB(tAcc, tPA[u & 1], mnmajor_desc(sSlot(it)), ID_ACC, u > 0);
-          tc_commit(bar(B_EMPTY + it % SLOTS));
-          if (u == nt - 1) tc_commit(bar(B_DONE));
+        if (tp < nt && tp - ts < 2) {                            // Phi^T(tp): its X items
+          bool ready = true;
+#pragma unroll
+          for (int j = 0; j < NX; ++j) {
+            const int it = tp * IPT + j;
+            ready = ready && mbar_try_wait(bar(B_FULL + it % SLOTS), (it / SLOTS) & 1);
+          }
+          if (ready) {
+            tc_fence_after();
+#pragma unroll
+            for (int j = 0; j < NX; ++j) {
+              const int it = tp * IPT + j;
+              issue_kmajor<D>(tD1[tp & 1], kmajor_desc(sW(j)), kmajor_desc(sSlot(it)), ID_PHI, j > 0);
+              tc_commit(bar(B_EMPTY + it % SLOTS));
+            }
+            tc_commit(bar(B_D1 + (tp & 1)));
+            ++tp;
+            did = true;
+          }
+        }
+        if (did) { polls = 0; t0 = 0; continue; }
+        // nothing was ready: the same bound as every other wait (the clock is looked at every 64 idle rounds)
+        if ((++polls & 63u) == 0u) {
+          const long long now = clock64();
+          if (t0 == 0) t0 = now;
+          if (*wc.abort != 0u || now - t0 > kWaitLimitCycles) {
+            *wc.abort = 1u;
+            atomicOr(wc.status, 1u);
+            ok = false;
+          }
         }
       }
     }
@@ -234,6 +273,7 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           for (int i = 0; i < IPT; ++i) mbar_arrive(bar(B_EMPTY + (t * IPT + i) % SLOTS));
       }
     }
+    named_barrier_arrive(2, K_FEATURE_THREADS + 64);           // the feature warps may reuse the ring for the partial S
   } else {
     // ------------------------------------------------------------ feature warps: lane of TMEM = feature
     // warp w works on TMEM lanes 32 * (w % 4) .. + 31 and on token columns 64 * (w / 4) .. + 63
@@ -288,26 +328,36 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       mbar_arrive(bar(B_PK + b));
     }
     if (ok) ok = mbar_wait_warp(bar(B_DONE), 0, wc);
-    // z of the two column halves is added through shared memory; every feature thread takes part in the barrier
+    // z of the two column halves is added through shared memory.  The partial S leaves through the ring: each
+    // thread puts its half row there (rows padded so that a warp's lanes hit different banks), then the row's
+    // owner hands the row to the copy engine as one contiguous piece - a row written straight from registers
+    // would cost one 32-byte sector per lane and instruction.  The ring is idle once the last product has
+    // completed and the gather warps (barrier 2) have read their last tile.  Every feature thread takes part in
+    // the barriers whatever its waits returned.
     if (hf == 1) sZ[f_local] = z0 + z1;
-    named_barrier_sync(1, K_FEATURE_THREADS);
+    named_barrier_sync(2, K_FEATURE_THREADS + 64);
+    uint8_t* stage = smem + L::RING_OFF + f_local * L::OUT_PITCH;
     if (ok) {
       tc_fence_after();
       constexpr int HALF = D / 2;                              // accumulator columns per warp
-      const size_t slot = (size_t)bh * p.n_chunks + chunk;
 #pragma unroll
       for (int c = 0; c < HALF / 32; ++c) {
         const int col = hf * HALF + c * 32;
         tmem_ld32(tAcc + lane_off + col, x);                   // warp-collective: also lanes beyond F take part
         tmem_ld_wait(x);
-        if (f < p.F) {
-          float* ps = p.part_s + (slot * p.F + f) * D + col;
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
-            *reinterpret_cast<uint4*>(ps + 4 * i) = make_uint4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]);
-        }
+        for (int i = 0; i < 8; ++i)
+          *reinterpret_cast<uint4*>(stage + (col + 4 * i) * 4) = make_uint4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]);
       }
-      if (hf == 0 && f < p.F) p.part_z[slot * p.F + f] = (z0 + z1) + sZ[f_local];
+      fence_proxy_async();
+    }
+    named_barrier_sync(1, K_FEATURE_THREADS);
+    if (ok && hf == 0 && f < p.F) {
+      const size_t slot = (size_t)bh * p.n_chunks + chunk;
+      bulk_store_1d(p.part_s + (slot * p.F + f) * D, smem_u32(stage), D * 4);
+      tma_store_commit();
+      p.part_z[slot * p.F + f] = (z0 + z1) + sZ[f_local];
+      tma_store_wait_all();
     }
   }
 

@@ -64,6 +64,15 @@ CONFIGS = {
                           block=(1, 6, 8), rate=16, seed=5000),
 }
 
+# The headline layer with wider feature maps ("Characterization of phi"; table of phi sizes): the paper's default
+# map, two layers d -> 2d -> 2d with polynomial degree 2, and a one-layer map of the same output width.
+VARIANTS = {
+    "wan81_paper_phi": Workload("wan81_paper_phi", B=1, H=12, d=128, F=256, grid=(21, 30, 52), block=(1, 6, 8),
+                                rate=8, seed=3100, layers=2, hidden=256),
+    "wan81_f256": Workload("wan81_f256", B=1, H=12, d=128, F=256, grid=(21, 30, 52), block=(1, 6, 8),
+                           rate=8, seed=3200),
+}
+
 STACK_RATES = (1, 4, 8, 16, 0)   # rate index -> R for the 30-layer block-rate stack
 STACK_LAYERS = 30
 
