@@ -176,6 +176,27 @@ AS_API as_status_t as_hybrid_attn_softmax_tokens(as_hybrid_attn_t h, int32_t* co
  * (Utility: no counterpart in the paper.) */
 AS_API as_status_t as_hybrid_attn_last_status(as_hybrid_attn_t h, void* cuda_stream);
 
+/* Gradient of the value-distillation loss w.r.t. the feature-map weights (section "Attention Distillation",
+ * value-distillation loss L = || y - y_hat ||_1; Algorithm 1: the student's update touches phi only).  To be
+ * called after `forward` with the same q, k, v, w on the same stream:
+ *   y_teacher  [B,H,N,d] bf16 device: the teacher block's attention output y
+ *   y_hat      [B,H,N,d] bf16 device: `out` of that forward
+ *   aux        [B,H,N,3] fp32 device: `aux` of that forward (required: c_i, den_S, den_L)
+ *   forward_workspace   the workspace of that forward, untouched since (it holds S and z)
+ *   dWq, dWk   [H,F,d] fp32 device, written: dL/dW_q and dL/dW_k, summed over the batch
+ *   loss       optional device float, written: L summed over every output element (must be NULL for a layer
+ *              without linear tokens, whose gradients are zero)
+ *   workspace  device scratch, 256-byte aligned, >= backward_workspace_bytes
+ * L = sum |y - y_hat|; q, k, v and y are constants of the step.  lambda_i (AS_STAB_EXACT: exp(-c_i)) and the softmax
+ * branch do not depend on the weights.  First version: fp32 on CUDA cores; one-layer feature maps with F == d and
+ * no bias, anything else returns AS_ERR_UNSUPPORTED.  Asynchronous on the stream; sums in a fixed order (no float
+ * atomics), so results are run-to-run identical. */
+AS_API as_status_t as_hybrid_attn_backward_workspace_bytes(as_hybrid_attn_t h, size_t* bytes);
+AS_API as_status_t as_hybrid_attn_backward_phi(as_hybrid_attn_t h, const void* q, const void* k, const void* v,
+                                               const as_phi_weights_t* w, const void* y_teacher, const void* y_hat,
+                                               const float* aux, const void* forward_workspace, float* dWq, float* dWk,
+                                               float* loss, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Test aid (no counterpart in the paper): enqueues a one-CTA kernel that waits, with the same bounded wait
  * every kernel of the library uses, on a barrier nobody arrives at; no copy and no tensor-core operation is
  * in flight.  After about `limit_cycles` SM clocks (1 .. 1e8) the wait gives up, the kernel returns and the

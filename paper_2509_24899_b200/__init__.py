@@ -89,6 +89,24 @@ class HybridAttention:
             None if biases is None else {n: t.data_ptr() for n, t in biases.items()})
         return out_host
 
+    def backward_phi(self, q, k, v, wq, wk, y_teacher, y_hat, aux, stream=None, want_loss=True):
+        """(dWq, dWk, loss) of the value-distillation loss sum |y_teacher - y_hat| w.r.t. the feature-map weights,
+        after `forward(..., out=y_hat, aux=aux)` on the same inputs (the handle's workspace still holds S and z)."""
+        import torch
+        B, H, N, d = self.shape
+        dwq = torch.empty(H, self.F, d, dtype=torch.float32, device="cuda")
+        dwk = torch.empty_like(dwq)
+        loss = torch.zeros(1, dtype=torch.float32, device="cuda") if want_loss else None
+        need = binding.as_hybrid_attn_backward_workspace_bytes(self._h)
+        if getattr(self, "_bws", None) is None or self._bws.numel() < need:
+            self._bws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        st = torch.cuda.current_stream() if stream is None else stream
+        binding.as_hybrid_attn_backward_phi(
+            self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), wq.data_ptr(), wk.data_ptr(), y_teacher.data_ptr(),
+            y_hat.data_ptr(), aux.data_ptr(), self.workspace().data_ptr(), dwq.data_ptr(), dwk.data_ptr(),
+            0 if loss is None else loss.data_ptr(), self._bws.data_ptr(), self._bws.numel(), st.cuda_stream)
+        return dwq, dwk, loss
+
     def linear_state(self, stream=None):
         """(S [B,H,F,d], z [B,H,F]) fp32 as left in the workspace by the last forward."""
         import torch

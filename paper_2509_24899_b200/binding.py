@@ -72,6 +72,10 @@ def lib() -> C.CDLL:
             "as_hybrid_attn_softmax_tokens": [H, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.c_int32],
             "as_hybrid_attn_last_status": [H, C.c_void_p],
             "as_hybrid_attn_debug_expire_wait": [H, C.c_int64, C.c_void_p],
+            "as_hybrid_attn_backward_workspace_bytes": [H, C.POINTER(C.c_size_t)],
+            "as_hybrid_attn_backward_phi": [H, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(as_phi_weights_t), C.c_void_p,
+                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                            C.c_void_p, C.c_size_t, C.c_void_p],
             "as_hybrid_attn_profile_enable": [H, C.c_int32],
             "as_hybrid_attn_profile_read": [H, C.POINTER(C.c_float), C.POINTER(C.c_int32)],
             "as_hybrid_attn_launch_count": [H, C.POINTER(C.c_uint64)],
@@ -189,6 +193,20 @@ def as_hybrid_attn_softmax_tokens(h, want_indices: bool = True):
 def as_hybrid_attn_last_status(h, stream_ptr) -> int:
     """Returns the status code instead of raising, so that callers can test for a time-out."""
     return lib().as_hybrid_attn_last_status(h, stream_ptr or None)
+
+
+def as_hybrid_attn_backward_workspace_bytes(h) -> int:
+    n = C.c_size_t()
+    _check(lib().as_hybrid_attn_backward_workspace_bytes(h, C.byref(n)), "as_hybrid_attn_backward_workspace_bytes")
+    return n.value
+
+
+def as_hybrid_attn_backward_phi(h, q_ptr, k_ptr, v_ptr, wq_ptr, wk_ptr, y_ptr, yhat_ptr, aux_ptr, fwd_ws_ptr, dwq_ptr,
+                                dwk_ptr, loss_ptr, ws_ptr, ws_bytes, stream_ptr) -> None:
+    """dL/dW_q, dL/dW_k (fp32 [H,F,d]) of L = sum |y - y_hat| after a forward; integer device addresses."""
+    _check(lib().as_hybrid_attn_backward_phi(h, q_ptr, k_ptr, v_ptr, _weights(wq_ptr, wk_ptr), y_ptr, yhat_ptr, aux_ptr,
+                                             fwd_ws_ptr, dwq_ptr, dwk_ptr, loss_ptr or None, ws_ptr, ws_bytes,
+                                             stream_ptr or None), "as_hybrid_attn_backward_phi")
 
 
 def as_hybrid_attn_debug_expire_wait(h, limit_cycles: int, stream_ptr) -> None:

@@ -162,6 +162,14 @@ def _draw(wl: Workload):
     return out
 
 
+def teacher_output(wl: Workload) -> np.ndarray:
+    """Stand-in for the teacher block's attention output y of the distillation step ("Attention Distillation"; the
+    real one needs the pretrained model): N(0, 1/4) draws [B, H, N, d] from a stream of its own (seed wl.seed + 77),
+    rounded to bf16; returns the bit patterns."""
+    rng = np.random.Generator(np.random.PCG64(wl.seed + 77))
+    return f32_to_bf16_bits(0.5 * rng.standard_normal((wl.B, wl.H, wl.N, wl.d), dtype=np.float32))
+
+
 WEIGHT_NAMES = ("wq", "wk", "wq2", "wk2", "bq1", "bk1", "bq2", "bk2")
 
 
