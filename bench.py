@@ -447,6 +447,75 @@ def run_ours(args, wl):
     return rc
 
 
+def run_seq_shard(args, wl):
+    """One layer with its TOKENS spread over the ranks (strong scaling): every rank holds a contiguous range of q, k, v
+    rows, runs the key stage, takes part in one all-reduce (S, z) and one all-gather (K_S, V_S) over NCCL, and runs the
+    query stage on its rows.  Prints one JSON line of its own; the headline line is the unsharded layer."""
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2509_24899_b200 import HybridAttention, seq_shard, workloads as W
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    class Alone:                                   # one rank: nothing to exchange
+        def all_reduce_sum(self, t):
+            return t
+
+        def all_gather_rows(self, t, rows_per_rank):
+            return t
+
+    # the layer's softmax tokens from the library's own token rule (a handle for the whole layer)
+    whole = HybridAttention.from_workload(wl)
+    idx = whole.softmax_indices()
+    whole.close()
+    op = seq_shard.SeqShardedAttention(wl.B, wl.H, wl.N, wl.d, idx, rank, world, comm=None if world > 1 else Alone(),
+                                       phi_dim=wl.F, poly_degree=wl.degree, phi_layers=wl.layers, phi_hidden=wl.hidden_width)
+    data = W.generate(wl)                          # the same layer on every rank; each keeps its rows
+    to_dev = lambda b: torch.from_numpy(b.view(np.int16)).cuda().view(torch.bfloat16)
+    rows = {k: to_dev(np.ascontiguousarray(data[k][:, :, op.n0:op.n1])) for k in ("q", "k", "v")}
+    wts = {k: to_dev(v) for k, v in data.items() if k not in ("q", "k", "v")}
+    extra = dict(wq2=wts.get("wq2"), wk2=wts.get("wk2"))
+    out = torch.empty_like(rows["q"])
+    stream = torch.cuda.current_stream()
+    step = lambda: op.forward(rows["q"], rows["k"], rows["v"], wts["wq"], wts["wk"], out=out, **extra)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    (ms,) = max_over_ranks([e0.elapsed_time(e1)], "cuda")
+    status = op.op.last_status()
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": wl.B * wl.N * args.steps / (ms * 1e-3), "unit": "tokens/s",
+                          "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
+                          "higher_is_better": True, "scaling": "strong", "dtype": "bf16", "data": "synthetic",
+                          "config": dict(config_of(wl, len(idx), world), parallelism="sp%d (token ranges; all-reduce of S, z and "
+                                         "all-gather of K_S, V_S per layer)" % world),
+                          "exchange_bytes_per_step": {"all_reduce": wl.B * wl.H * wl.F * (wl.d + 1) * 4,
+                                                      "all_gather": 2 * wl.B * wl.H * len(idx) * wl.d * 2},
+                          "device_status": status}))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0 if status == 0 else 1
+
+
 def run_stack(args):
     """The 30-layer block-rate stack: one timed layer per distinct rate, per-layer and summed time against
     all layers running full softmax (rate 1).  Prints one JSON line of its own; not the headline line."""
@@ -509,6 +578,9 @@ def main():
                     help="kernel path: tcgen05 tensor-core kernels (default) or the fp32 CUDA-core check path")
     ap.add_argument("--sustained-s", type=float, default=2.0,
                     help="length in seconds of the second, power-capped timed region (0 = none)")
+    ap.add_argument("--shard", default="batch", choices=["batch", "seq"],
+                    help="batch: every rank its own layer input (the headline, weak scaling); seq: one layer with its "
+                         "tokens spread over the ranks (strong scaling, two NCCL exchanges per layer)")
     ap.add_argument("--skip-extras", action="store_true",
                     help="only the device-timed steps (for profiler runs): no e2e, no CPU baseline")
     args = ap.parse_args()
@@ -523,6 +595,8 @@ def main():
         wl = W.CONFIGS[args.workload]
     if args.impl == "reference":
         return run_reference(args, wl)
+    if args.shard == "seq":
+        return run_seq_shard(args, wl)
     return run_ours(args, wl)
 
 

@@ -176,6 +176,29 @@ AS_API as_status_t as_hybrid_attn_softmax_tokens(as_hybrid_attn_t h, int32_t* co
  * (Utility: no counterpart in the paper.) */
 AS_API as_status_t as_hybrid_attn_last_status(as_hybrid_attn_t h, void* cuda_stream);
 
+/* The forward pass in two stages, for a layer whose TOKENS are spread over several GPUs (sequence sharding).
+ * The linear state is a sum over keys that does not depend on the query ("Preliminaries: Linear Attention": the two
+ * sums can be precomputed), so partial states of token ranges add up, and the softmax tokens of the ranges
+ * concatenate; a query then needs only the summed state and the gathered softmax keys (hybrid equation).  Each
+ * rank creates a handle for ITS token range (N = tokens of the range, softmax_idx = the range's softmax tokens,
+ * counted from the range's start) and runs:
+ *   key_pass      k, v [B,H,N,d] of the range -> in `workspace`: the range's softmax keys and values K_S, V_S
+ *                 [B*H, n_softmax, d] bf16 and its partial state S [B*H,F,d], z [B*H,F] fp32, at the byte offsets
+ *                 `workspace_offsets` returns.  A range without linear tokens is left alone (its keys are k, v
+ *                 themselves, its state is zero); a range without softmax tokens leaves no K_S, V_S.
+ *   (the caller sums S, z over the ranks and gathers K_S, V_S in rank order, each into local memory)
+ *   query_pass    q [B,H,N,d] of the range, the gathered keys ks, vs [B*H, n_keys, d] bf16 (n_keys may be 0), the
+ *                 summed S, z (both NULL when no rank has linear tokens) -> out [B,H,N,d] (, aux).  `workspace` is
+ *                 scratch of at least workspace_bytes again (it receives S as a bf16 operand); a handle whose own
+ *                 range has no linear tokens cannot take a state (AS_ERR_UNSUPPORTED: its workspace has no room).
+ * Both are asynchronous on the stream, allocate nothing, and share every rule of `forward`. */
+AS_API as_status_t as_hybrid_attn_key_pass(as_hybrid_attn_t h, const void* k, const void* v, const as_phi_weights_t* w,
+                                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+AS_API as_status_t as_hybrid_attn_workspace_offsets(as_hybrid_attn_t h, size_t* ks, size_t* vs, size_t* S, size_t* z);
+AS_API as_status_t as_hybrid_attn_query_pass(as_hybrid_attn_t h, const void* q, const as_phi_weights_t* w, const void* ks,
+                                             const void* vs, int32_t n_keys, const float* S, const float* z, void* out,
+                                             float* aux, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Gradient of the value-distillation loss w.r.t. the feature-map weights (section "Attention Distillation",
  * value-distillation loss L = || y - y_hat ||_1; Algorithm 1: the student's update touches phi only).  To be
  * called after `forward` with the same q, k, v, w on the same stream:

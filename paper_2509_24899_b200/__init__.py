@@ -89,6 +89,49 @@ class HybridAttention:
             None if biases is None else {n: t.data_ptr() for n, t in biases.items()})
         return out_host
 
+    def key_pass(self, k, v, wq=None, wk=None, stream=None, wq2=None, wk2=None, biases=None):
+        """First stage of a sequence-sharded forward on this handle's token range.  Returns (K_S, V_S, S, z): the
+        range's softmax keys / values [B*H, n_softmax, d] (bf16) and its partial linear state [B*H, F, d], [B*H, F]
+        (fp32).  K_S, V_S, S, z are views into the handle's workspace (k, v themselves and zeros for a range without
+        linear tokens)."""
+        import torch
+        B, H, N, d = self.shape
+        BH = B * H
+        if self.n_softmax == N:
+            return (k.reshape(BH, N, d), v.reshape(BH, N, d),
+                    torch.zeros(BH, self.F, d, dtype=torch.float32, device=k.device),
+                    torch.zeros(BH, self.F, dtype=torch.float32, device=k.device))
+        ws = self.workspace()
+        st = torch.cuda.current_stream() if stream is None else stream
+        binding.as_hybrid_attn_key_pass(
+            self._h, k.data_ptr(), v.data_ptr(), 0 if wq is None else wq.data_ptr(), 0 if wk is None else wk.data_ptr(),
+            ws.data_ptr(), ws.numel(), st.cuda_stream, 0 if wq2 is None else wq2.data_ptr(),
+            0 if wk2 is None else wk2.data_ptr(), None if biases is None else {n: t.data_ptr() for n, t in biases.items()})
+        o_ks, o_vs, o_S, o_z = binding.as_hybrid_attn_workspace_offsets(self._h)
+        n_s = self.n_softmax
+        view = lambda off, count, dtype, shape: ws[off:off + count * dtype.itemsize].view(dtype).view(*shape)
+        ks = view(o_ks, BH * n_s * d, torch.bfloat16, (BH, n_s, d))
+        vs = view(o_vs, BH * n_s * d, torch.bfloat16, (BH, n_s, d))
+        return ks, vs, view(o_S, BH * self.F * d, torch.float32, (BH, self.F, d)), view(o_z, BH * self.F, torch.float32, (BH, self.F))
+
+    def query_pass(self, q, wq, wk, ks, vs, S, z, out=None, aux=None, stream=None, wq2=None, wk2=None, biases=None):
+        """Second stage: this range's queries against the gathered softmax keys ks, vs [B*H, n_keys, d] and the summed
+        state S, z (None, None when the layer has no linear tokens).  Returns the range's output rows."""
+        import torch
+        if out is None:
+            out = torch.empty_like(q)
+        ws = self.workspace()
+        st = torch.cuda.current_stream() if stream is None else stream
+        n_keys = 0 if ks is None else ks.shape[1]
+        binding.as_hybrid_attn_query_pass(
+            self._h, q.data_ptr(), 0 if wq is None else wq.data_ptr(), 0 if wk is None else wk.data_ptr(),
+            ks.data_ptr() if n_keys else 0, vs.data_ptr() if n_keys else 0, n_keys,
+            0 if S is None else S.data_ptr(), 0 if z is None else z.data_ptr(), out.data_ptr(),
+            0 if aux is None else aux.data_ptr(), ws.data_ptr(), ws.numel(), st.cuda_stream,
+            0 if wq2 is None else wq2.data_ptr(), 0 if wk2 is None else wk2.data_ptr(),
+            None if biases is None else {n: t.data_ptr() for n, t in biases.items()})
+        return out
+
     def backward_phi(self, q, k, v, wq, wk, y_teacher, y_hat, aux, stream=None, want_loss=True):
         """(dWq, dWk, loss) of the value-distillation loss sum |y_teacher - y_hat| w.r.t. the feature-map weights,
         after `forward(..., out=y_hat, aux=aux)` on the same inputs (the handle's workspace still holds S and z)."""

@@ -72,6 +72,10 @@ def lib() -> C.CDLL:
             "as_hybrid_attn_softmax_tokens": [H, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.c_int32],
             "as_hybrid_attn_last_status": [H, C.c_void_p],
             "as_hybrid_attn_debug_expire_wait": [H, C.c_int64, C.c_void_p],
+            "as_hybrid_attn_key_pass": [H, C.c_void_p, C.c_void_p, C.POINTER(as_phi_weights_t), C.c_void_p, C.c_size_t, C.c_void_p],
+            "as_hybrid_attn_workspace_offsets": [H] + [C.POINTER(C.c_size_t)] * 4,
+            "as_hybrid_attn_query_pass": [H, C.c_void_p, C.POINTER(as_phi_weights_t), C.c_void_p, C.c_void_p, C.c_int32,
+                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p],
             "as_hybrid_attn_backward_workspace_bytes": [H, C.POINTER(C.c_size_t)],
             "as_hybrid_attn_backward_phi": [H, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(as_phi_weights_t), C.c_void_p,
                                             C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -193,6 +197,29 @@ def as_hybrid_attn_softmax_tokens(h, want_indices: bool = True):
 def as_hybrid_attn_last_status(h, stream_ptr) -> int:
     """Returns the status code instead of raising, so that callers can test for a time-out."""
     return lib().as_hybrid_attn_last_status(h, stream_ptr or None)
+
+
+def as_hybrid_attn_key_pass(h, k_ptr, v_ptr, wq_ptr, wk_ptr, ws_ptr, ws_bytes, stream_ptr, wq2_ptr=0, wk2_ptr=0,
+                            biases=None) -> None:
+    """First stage of a sequence-sharded forward: this range's K_S, V_S and partial S, z into the workspace."""
+    _check(lib().as_hybrid_attn_key_pass(h, k_ptr, v_ptr, _weights(wq_ptr, wk_ptr, wq2_ptr, wk2_ptr, biases), ws_ptr,
+                                         ws_bytes, stream_ptr or None), "as_hybrid_attn_key_pass")
+
+
+def as_hybrid_attn_workspace_offsets(h):
+    """Byte offsets (K_S, V_S, S, z) inside the workspace."""
+    o = [C.c_size_t() for _ in range(4)]
+    _check(lib().as_hybrid_attn_workspace_offsets(h, *[C.byref(x) for x in o]), "as_hybrid_attn_workspace_offsets")
+    return tuple(x.value for x in o)
+
+
+def as_hybrid_attn_query_pass(h, q_ptr, wq_ptr, wk_ptr, ks_ptr, vs_ptr, n_keys, S_ptr, z_ptr, out_ptr, aux_ptr, ws_ptr,
+                              ws_bytes, stream_ptr, wq2_ptr=0, wk2_ptr=0, biases=None) -> None:
+    """Second stage: this range's queries against the gathered keys and the summed state."""
+    _check(lib().as_hybrid_attn_query_pass(h, q_ptr, _weights(wq_ptr, wk_ptr, wq2_ptr, wk2_ptr, biases), ks_ptr or None,
+                                           vs_ptr or None, int(n_keys), S_ptr or None, z_ptr or None, out_ptr,
+                                           aux_ptr or None, ws_ptr, ws_bytes, stream_ptr or None),
+           "as_hybrid_attn_query_pass")
 
 
 def as_hybrid_attn_backward_workspace_bytes(h) -> int:

@@ -107,9 +107,18 @@ struct ProfileScope {
 
 }  // namespace
 
+// Keys and linear state handed to the query stage from outside (sequence sharding: gathered / summed over ranks).
+struct as_ext_state {
+  const void *ks, *vs;         // [B*H, n_keys, d] bf16
+  int n_keys;
+  const float *S, *z;          // [B*H, F, d], [B*H, F] fp32; NULL: no linear tokens anywhere
+};
+enum { AS_STAGE_KEYS = 1, AS_STAGE_QUERIES = 2 };
+
 static as_status_t launch_heads(as_hybrid_attn_t h, const void* q, const void* k, const void* v,
                                 const as_phi_weights_t* w, void* out, float* aux, char* ws, cudaStream_t st,
-                                int first, int count, int nb, int nh);
+                                int first, int count, int nb, int nh, int stages = AS_STAGE_KEYS | AS_STAGE_QUERIES,
+                                const as_ext_state* ext = nullptr);
 
 // A handle works on the device it was created on: its tables live there and the kernels' shared-memory opt-in
 // was made there.
@@ -262,9 +271,10 @@ as_status_t as_hybrid_attn_forward(as_hybrid_attn_t h, const void* q, const void
 // their place in the full [B*H] arrays, so linear_state sees every pair afterwards.
 static as_status_t launch_heads(as_hybrid_attn_t h, const void* q, const void* k, const void* v,
                                 const as_phi_weights_t* w, void* out, float* aux, char* ws, cudaStream_t st,
-                                int first, int count, int nb, int nh) {
+                                int first, int count, int nb, int nh, int stages, const as_ext_state* ext) {
   const auto& d = h->desc;
-  const bool lin = h->n_l > 0;
+  // with outside state the linear branch exists when a state is given, whatever this handle's own tokens are
+  const bool lin = ext ? (ext->S != nullptr) : (h->n_l > 0);
   const int head0 = first % d.H;                 // the run's first head: where its weights start
   const size_t F = d.phi_dim, dd = d.d;
   (void)count;
@@ -299,9 +309,21 @@ static as_status_t launch_heads(as_hybrid_attn_t h, const void* q, const void* k
   a.B = nb; a.H = nh; a.N = d.N; a.d = d.d; a.F = d.phi_dim; a.P = d.poly_degree;
   a.n_s = h->n_s; a.n_l = h->n_l; a.n_chunks = h->n_chunks; a.chunk_tiles = h->chunk_tiles;
   a.scale = h->scale; a.stab_mode = d.stab_mode;
-
   const bool simt = d.kernel_path == AS_PATH_SIMT;
   cudaError_t e = cudaSuccess;
+  if (ext) {
+    // query stage on gathered keys and a summed state: S as the bf16 operand into this workspace
+    a.ks = (const __nv_bfloat16*)ext->ks; a.vs = (const __nv_bfloat16*)ext->vs;
+    a.ks_w = a.vs_w = nullptr;
+    a.n_s = ext->n_keys; a.n_l = lin ? 1 : 0;
+    if (lin) {
+      a.S = const_cast<float*>(ext->S); a.z = const_cast<float*>(ext->z);
+      { ProfileScope p(h, st, AS_KERNEL_REDUCE);
+        e = as_round_state(a, st); }
+      if (e != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
+    }
+  }
+  if (!(stages & AS_STAGE_KEYS)) goto queries;
   if (two) {
     { ProfileScope p(h, st, AS_KERNEL_KPASS);     // counted with the K pass: it feeds it
       e = as_tensor_phi1(a, st); }
@@ -315,6 +337,8 @@ static as_status_t launch_heads(as_hybrid_attn_t h, const void* q, const void* k
       e = as_reduce_state(a, st); }
     if (e != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
   }
+queries:
+  if (!(stages & AS_STAGE_QUERIES)) return AS_OK;
   { ProfileScope p(h, st, AS_KERNEL_QPASS);
     e = simt ? as_simt_qpass(a, st) : as_tensor_qpass(a, st); }
   if (e != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
@@ -414,6 +438,50 @@ as_status_t as_hybrid_attn_last_status(as_hybrid_attn_t h, void* cuda_stream) {
   }
   if (word != 0 && cudaMemset(h->d_status, 0, 4) != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
   return (word & AS_DEV_TIMEOUT) ? AS_ERR_DEVICE_TIMEOUT : AS_OK;
+}
+
+as_status_t as_hybrid_attn_key_pass(as_hybrid_attn_t h, const void* k, const void* v, const as_phi_weights_t* w,
+                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!h || !k || !v) return AS_ERR_INVALID_ARG;
+  if (!on_handle_device(h)) return AS_ERR_INVALID_ARG;
+  const auto& d = h->desc;
+  const as_status_t ws_ok = check_weights(h, w);
+  if (ws_ok != AS_OK) return ws_ok;
+  if (((uintptr_t)k | (uintptr_t)v) & 15) return AS_ERR_INVALID_ARG;
+  if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < h->ws.total) return AS_ERR_WORKSPACE;
+  if (h->n_l == 0) return AS_OK;                  // nothing to sum and nothing to compact: the keys are k, v themselves
+  return launch_heads(h, k, k, v, w, nullptr, nullptr, (char*)workspace, (cudaStream_t)cuda_stream, 0, d.B * d.H, d.B, d.H,
+                      AS_STAGE_KEYS, nullptr);
+}
+
+as_status_t as_hybrid_attn_workspace_offsets(as_hybrid_attn_t h, size_t* ks, size_t* vs, size_t* S, size_t* z) {
+  if (!h || !ks || !vs || !S || !z) return AS_ERR_INVALID_ARG;
+  *ks = h->ws.ks; *vs = h->ws.vs; *S = h->ws.S; *z = h->ws.z;
+  return AS_OK;
+}
+
+as_status_t as_hybrid_attn_query_pass(as_hybrid_attn_t h, const void* q, const as_phi_weights_t* w, const void* ks,
+                                      const void* vs, int32_t n_keys, const float* S, const float* z, void* out,
+                                      float* aux, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!h || !q || !out || n_keys < 0 || (n_keys > 0 && (!ks || !vs)) || ((S == nullptr) != (z == nullptr))) return AS_ERR_INVALID_ARG;
+  if (n_keys == 0 && !S) return AS_ERR_INVALID_ARG;            // nothing to attend to
+  if (!on_handle_device(h)) return AS_ERR_INVALID_ARG;
+  const auto& d = h->desc;
+  if (S) {
+    if (!w || !w->wq1) return AS_ERR_INVALID_ARG;
+    if (d.phi_layers == 2 && !w->wq2) return AS_ERR_INVALID_ARG;
+    if (((uintptr_t)w->wq1 | (uintptr_t)w->wq2) & 15) return AS_ERR_INVALID_ARG;
+    if (((uintptr_t)w->bq1 | (uintptr_t)w->bq2) & 3) return AS_ERR_INVALID_ARG;
+  }
+  if (((uintptr_t)q | (uintptr_t)out | (uintptr_t)ks | (uintptr_t)vs | (uintptr_t)S) & 15) return AS_ERR_INVALID_ARG;
+  if (aux && ((uintptr_t)aux & 3)) return AS_ERR_INVALID_ARG;
+  if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < h->ws.total) return AS_ERR_WORKSPACE;
+  // the workspace must have room for the bf16 copy of S even when this handle's own tokens are all softmax tokens
+  if (S && h->n_l == 0) return AS_ERR_UNSUPPORTED;
+  const as_ext_state ext{ks, vs, n_keys, S, z};
+  as_phi_weights_t none{};
+  return launch_heads(h, q, q, q, w ? w : &none, out, aux, (char*)workspace, (cudaStream_t)cuda_stream, 0, d.B * d.H, d.B, d.H,
+                      AS_STAGE_QUERIES, &ext);
 }
 
 as_status_t as_hybrid_attn_debug_expire_wait(as_hybrid_attn_t h, int64_t limit_cycles, void* cuda_stream) {

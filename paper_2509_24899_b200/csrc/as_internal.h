@@ -73,6 +73,8 @@ struct as_hybrid_attn_s {
 cudaError_t as_simt_kpass(const as_launch_args& a, cudaStream_t st);
 cudaError_t as_simt_qpass(const as_launch_args& a, cudaStream_t st);
 cudaError_t as_reduce_state(const as_launch_args& a, cudaStream_t st);
+// Sb = bf16(S) for a state that came from outside (the Q pass reads S as a bf16 operand).
+cudaError_t as_round_state(const as_launch_args& a, cudaStream_t st);
 cudaError_t as_tensor_kpass(const as_launch_args& a, cudaStream_t st);
 cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st);
 // First layer of a two-layer feature map for the keys: h1k = relu(k W_k1^T + b_k1).

@@ -116,6 +116,11 @@ __global__ void reduce_state_kernel(as_launch_args a) {
   }
 }
 
+__global__ void round_state_kernel(const float* S, __nv_bfloat16* Sb, size_t n) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) Sb[i] = __float2bfloat16_rn(S[i]);
+}
+
 constexpr int QP_WARPS = 8;
 
 // Q pass: one warp per query row.  Online softmax over the softmax tokens, then the linear
@@ -253,6 +258,12 @@ cudaError_t as_reduce_state(const as_launch_args& a, cudaStream_t st) {
   const int n = a.F * a.d + a.F;
   dim3 grid((n + 255) / 256, a.B * a.H);
   reduce_state_kernel<<<grid, 256, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t as_round_state(const as_launch_args& a, cudaStream_t st) {
+  const size_t n = (size_t)a.B * a.H * a.F * a.d;
+  round_state_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a.S, a.Sb, n);
   return cudaGetLastError();
 }
 
