@@ -740,6 +740,197 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
   return true;
 }
 
+// ---------------------------------------------------------------- layers without softmax tokens (rate 0)
+// With no key loop a unit is: Phi = Q W^T, phi_q, O = phi_q S, y = O / (phi_q . z), store.  The tensor pipe has
+// little to do and the kernel is bound by how fast the threads turn rows around, so this variant of the kernel runs
+// SIXTEEN compute warps: each 128-row group is worked on by two warps per TMEM lane quadrant, each taking one half of
+// the columns of a row (features on the way in, output columns on the way out).  Producer and issuing threads are the
+// ones of the general kernel; a row's two threads add their shares of phi_q . z through shared memory.
+constexpr int QL_THREADS = 608;          // warps 0-15: compute (group = bit 2, quadrant = bits 0-1, column half = bit 3);
+                                         // warp 16: TMA; warps 17, 18: MMA issuers
+
+template <int D, bool GEN>
+__device__ __noinline__ bool q_linear_unit(const QParams& p, const QCtx& c, const CUtensorMap* tmO, uint8_t* smem, float* sDl, int u) {
+  using R = QRing<D>;
+  using L = QLayout<D>;
+  const R q(p, c);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = (warp >> 2) & 1, quad = warp & 3, hf = warp >> 3;
+  const int r = quad * 32 + lane;                   // row inside the group's 128-row tile
+  const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
+  const uint32_t tSg = q.tS(g) + lane_off, tOg = q.tO(g) + lane_off;
+  uint8_t* sPg = smem + L::P_OFF + g * L::PTILE;    // phi_q, then the output rows
+  float* dl_slot = sDl + g * 128 + r;
+  const int ps = u * q.n_s, ppf = u * q.n_pf;
+  const int fcw = D == 128 ? 128 : p.fcw;           // width of a feature chunk; this thread takes columns [hf, hf + 1) * half
+  const int half = fcw / 2;
+  const QUnit un = q_unit(p, u);
+  const int bh = un.w / p.nx, row = un.row0 + g * 128 + r;
+  const int part = p.F / p.P;
+  uint32_t x[32];
+  float dl = 0.f;
+  for (int ch = 0; ch < q.fc; ++ch) {
+    if (!q.wait(R::B_S + g, ps + ch)) return false;
+    tc_fence_after();
+    // the P tile may be written once the product that read it has completed and the previous unit's output store
+    // has been read out (the stores are issued by the warps of column half 0)
+    if (hf == 0 && lane == 0) tma_store_wait_read();
+    if (ppf + ch > 0 && !q.wait(R::B_PF + g, ppf + ch - 1)) return false;
+    named_barrier_sync(1 + g, 256);
+    const float2* zrow = reinterpret_cast<const float2*>(p.z + (size_t)bh * p.F + ch * 128 + hf * half);
+    const uint32_t* brow = nullptr;
+    if (GEN && p.b2 != nullptr) brow = reinterpret_cast<const uint32_t*>(p.b2 + (size_t)(bh % p.H) * p.F + ch * 128 + hf * half);
+    float dl0 = 0.f, dl1 = 0.f;
+#pragma unroll
+    for (int cc = 0; cc < 2; ++cc) {
+      if (cc * 32 < half) {
+        const int col = hf * half + cc * 32;
+        tmem_ld32(tSg + col, x);
+        tmem_ld_wait(x);
+        const int pw = min((ch * 128 + col) / part, p.P - 1);
+        uint32_t wd[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float a0 = __uint_as_float(x[2 * i]), a1 = __uint_as_float(x[2 * i + 1]);
+          if (GEN && brow != nullptr) {
+            const uint32_t bb = __ldg(brow + cc * 16 + i);
+            a0 += __uint_as_float(bb << 16);
+            a1 += __uint_as_float(bb & 0xffff0000u);
+          }
+          a0 = fmaxf(a0, 0.f); a1 = fmaxf(a1, 0.f);
+          float r0 = a0, r1 = a1;
+          if (pw >= 1) { r0 *= a0; r1 *= a1; }
+          if (GEN) {
+            if (pw >= 2) { r0 *= a0; r1 *= a1; }
+            if (pw >= 3) { r0 *= a0; r1 *= a1; }
+          }
+          wd[i] = pack_bf16(r0, r1);
+          const float2 zz = __ldg(zrow + cc * 16 + i);
+          dl0 = fmaf(__uint_as_float(wd[i] << 16), zz.x, dl0);
+          dl1 = fmaf(__uint_as_float(wd[i] & 0xffff0000u), zz.y, dl1);
+        }
+        store_row_chunk(sPg, r, col, wd);
+      }
+    }
+    dl += dl0 + dl1;
+    tc_fence_before();
+    mbar_arrive(q.bar(R::B_SF + g));                 // the next product into the score columns may follow
+    fence_proxy_async();
+    mbar_arrive(q.bar(R::B_P + g));
+  }
+  // the row's denominator: both column halves' shares of phi_q . z
+  if (hf == 1) *dl_slot = dl;
+  named_barrier_sync(1 + g, 256);
+  if (hf == 0) dl += *dl_slot;
+  named_barrier_sync(1 + g, 256);
+  if (hf == 0) *dl_slot = dl;
+  if (!q.wait(R::B_O + g, u)) return false;          // (the products run meanwhile)
+  named_barrier_sync(1 + g, 256);
+  const float den = *dl_slot;
+  tc_fence_after();
+  const float inv = 1.f / den;
+  const int ohalf = D / 2;                           // output columns per thread
+#pragma unroll
+  for (int cc = 0; cc < 2; ++cc) {
+    if (cc * 32 < ohalf) {
+      const int col = hf * ohalf + cc * 32;
+      tmem_ld32(tOg + col, x);
+      tmem_ld_wait(x);
+      uint32_t wd[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) wd[i] = pack_bf16(__uint_as_float(x[2 * i]) * inv, __uint_as_float(x[2 * i + 1]) * inv);
+      store_row_chunk(sPg, r, col, wd);
+    }
+  }
+  fence_proxy_async();
+  tc_fence_before();
+  named_barrier_sync(1 + g, 256);                    // both halves of every row are staged
+  const int wrow0 = row - lane;
+  if (hf == 0 && lane == 0 && wrow0 < p.N) {
+#pragma unroll
+    for (int b = 0; b < D / 64; ++b)
+      tma_store_3d(tmO, smem_u32(sPg) + b * BOX_BYTES + quad * 32 * 128, b * 64, wrow0, bh);
+    tma_store_commit();
+  }
+  if (hf == 0 && p.aux != nullptr && row < p.N) {
+    float* ap = p.aux + ((size_t)bh * p.N + row) * 3;
+    ap[0] = 0.f; ap[1] = 0.f; ap[2] = den;
+  }
+  return true;
+}
+
+template <int D, bool GEN>
+__global__ void __launch_bounds__(QL_THREADS, 1)
+qlin_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmW,
+            const __grid_constant__ CUtensorMap tmSt, const __grid_constant__ CUtensorMap tmO, const __grid_constant__ QParams p) {
+  using L = QLayout<D>;
+  using R = QRing<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::BAR_OFF + 8 * R::B_COUNT);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::BAR_OFF + 8 * R::B_COUNT + 4);
+  auto bar = [&](int i) { return sbase + L::BAR_OFF + 8 * i; };
+  const int warp = threadIdx.x >> 5;
+  __shared__ float sDl[2 * 128];                     // per group and row: share of phi_q . z, then the denominator
+
+  __shared__ uint32_t s_skip;
+  if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile uint32_t*>(p.status);
+  __syncthreads();
+  if (s_skip != 0u) return;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0u;
+    mbar_init(bar(R::B_Q0), 1); mbar_init(bar(R::B_Q0 + 1), 1);
+    for (int s = 0; s < KV_STAGES; ++s) { mbar_init(bar(R::B_FULL + s), 1); mbar_init(bar(R::B_EMPTY + s), 1); }
+    for (int g = 0; g < 2; ++g) {
+      mbar_init(bar(R::B_S + g), 1); mbar_init(bar(R::B_SF + g), 256); mbar_init(bar(R::B_P + g), 256);
+      mbar_init(bar(R::B_PF + g), 1); mbar_init(bar(R::B_O + g), 1); mbar_init(bar(R::B_QF + g), 1);
+      mbar_init(bar(R::B_H + g), 128);
+    }
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 17) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const QCtx c{sbase, *tmem_slot, WaitCtx{p.status, abort_flag}};
+  const int n_mine = q_units_of_cta(p);
+
+  if (warp == 16) {
+    if ((threadIdx.x & 31) == 0) { tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmW); tma_prefetch_desc(&tmSt); tma_prefetch_desc(&tmO); }
+    for (int u = 0; u < n_mine; ++u)
+      if (!q_produce_unit<D, false, GEN>(p, c, &tmQ, &tmQ, &tmQ, &tmW, &tmSt, &tmW, u)) break;
+  } else if (warp == 17) {
+    if ((threadIdx.x & 31) == 0) {
+      for (int u = 0; u < n_mine; ++u)
+        if (!q_score_unit<D, false, GEN>(p, c, u)) break;
+    }
+    __syncwarp();
+  } else if (warp == 18) {
+    if ((threadIdx.x & 31) == 0) {
+      for (int u = 0; u < n_mine; ++u)
+        if (!q_accum_unit<D, false, GEN>(p, c, u)) break;
+    }
+    __syncwarp();
+  } else {
+    const int g = (warp >> 2) & 1;
+    // a unit worked on by one group only (a left-over half) is the CTA's last one: group 1 stops before it
+    const int n_grp = (n_mine > p.n_rounds && p.split_last && g == 1) ? p.n_rounds : n_mine;
+    for (int u = 0; u < n_grp; ++u)
+      if (!q_linear_unit<D, GEN>(p, c, &tmO, smem, sDl, u)) break;
+    if ((threadIdx.x & 31) == 0) tma_store_wait_all();
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 17) {
+    tc_fence_after();
+    tmem_dealloc(c.tmem, 512);
+  }
+}
+
 template <int D, bool TWO, bool GEN>
 __global__ void __launch_bounds__(Q_THREADS, 1)
 qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -826,6 +1017,10 @@ cudaError_t as_tensor_init_qpass() {
   if ((e = opt_in_smem(qpass_kernel<64, false, true>, QLayout<64>::TOTAL)) != cudaSuccess) return e;
   if ((e = opt_in_smem(qpass_kernel<64, true, false>, QLayout<64>::TOTAL)) != cudaSuccess) return e;
   if ((e = opt_in_smem(qpass_kernel<64, true, true>, QLayout<64>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(qlin_kernel<128, false>, QLayout<128>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(qlin_kernel<128, true>, QLayout<128>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(qlin_kernel<64, false>, QLayout<64>::TOTAL)) != cudaSuccess) return e;
+  if ((e = opt_in_smem(qlin_kernel<64, true>, QLayout<64>::TOTAL)) != cudaSuccess) return e;
   return cudaSuccess;
 }
 
@@ -874,6 +1069,17 @@ cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st) {
   p.split_last = (left > 0 && 2 * left <= (int)grid.x) ? 1 : 0;
   // the general kernels carry the bias and the powers beyond 2; the common case does without them
   const bool gen = lin && (a.P > 2 || p.b1 != nullptr || p.b2 != nullptr);
+  if (p.nkv == 0 && lin && !two) {
+    // no softmax tokens, one-layer map: the variant with sixteen compute warps
+    if (a.d == 128) {
+      if (gen) qlin_kernel<128, true><<<grid, QL_THREADS, QLayout<128>::TOTAL, st>>>(tmQ, tmW, tmSt, tmO, p);
+      else qlin_kernel<128, false><<<grid, QL_THREADS, QLayout<128>::TOTAL, st>>>(tmQ, tmW, tmSt, tmO, p);
+    } else {
+      if (gen) qlin_kernel<64, true><<<grid, QL_THREADS, QLayout<64>::TOTAL, st>>>(tmQ, tmW, tmSt, tmO, p);
+      else qlin_kernel<64, false><<<grid, QL_THREADS, QLayout<64>::TOTAL, st>>>(tmQ, tmW, tmSt, tmO, p);
+    }
+    return cudaGetLastError();
+  }
 #define AS_LAUNCH_Q(D_, TWO_, GEN_) \
   qpass_kernel<D_, TWO_, GEN_><<<grid, Q_THREADS, QLayout<D_>::TOTAL, st>>>(tmQ, tmK, tmV, tmW, tmSt, tmW1, tmO, p)
   if (a.d == 128) {
