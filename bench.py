@@ -26,7 +26,7 @@ sys.path.insert(0, ROOT)
 
 METRIC = "hybrid-attn fwd tokens/s per layer at N=32760 (12x128 heads); % of bf16 tensor peak"
 
-KERNEL_SOURCES = ("tensor_qpass.cu", "tensor_kpass.cu", "tensor_common.cuh", "sm100_ptx.cuh", "sm100_tmem_wide.cuh")
+KERNEL_SOURCES = ("tensor_qpass.cu", "tensor_qstream.cu", "tensor_kpass.cu", "tensor_common.cuh", "sm100_ptx.cuh", "sm100_tmem_wide.cuh")
 
 
 def kernel_source_digest(names=KERNEL_SOURCES):

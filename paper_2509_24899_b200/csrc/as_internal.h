@@ -77,6 +77,10 @@ cudaError_t as_reduce_state(const as_launch_args& a, cudaStream_t st);
 cudaError_t as_round_state(const as_launch_args& a, cudaStream_t st);
 cudaError_t as_tensor_kpass(const as_launch_args& a, cudaStream_t st);
 cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st);
+// Query stage of layers without softmax tokens in its streaming form (one-layer map, F = d = 128, no bias, degree
+// <= 2): whether it covers the launch, and the launch itself.  as_tensor_qpass dispatches to it.
+bool as_tensor_qstream_handles(const as_launch_args& a);
+cudaError_t as_tensor_qstream(const as_launch_args& a, cudaStream_t st);
 // First layer of a two-layer feature map for the keys: h1k = relu(k W_k1^T + b_k1).
 cudaError_t as_tensor_phi1(const as_launch_args& a, cudaStream_t st);
 // One-time set-up of the tensor path on the current device (driver entry points, smem opt-in).

@@ -74,3 +74,4 @@ cudaError_t opt_in_smem(K kernel, int bytes) {
 // Per-device set-up of each translation unit's kernels (shared-memory opt-in).
 cudaError_t as_tensor_init_qpass();
 cudaError_t as_tensor_init_kpass();
+cudaError_t as_tensor_init_qstream();

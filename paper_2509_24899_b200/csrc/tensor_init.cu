@@ -66,5 +66,6 @@ cudaError_t as_tensor_init() {
   // shared-memory opt-in is per device; cheap enough to repeat
   cudaError_t e;
   if ((e = as_tensor_init_qpass()) != cudaSuccess) return e;
-  return as_tensor_init_kpass();
+  if ((e = as_tensor_init_kpass()) != cudaSuccess) return e;
+  return as_tensor_init_qstream();
 }

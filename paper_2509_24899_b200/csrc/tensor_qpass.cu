@@ -1025,6 +1025,7 @@ cudaError_t as_tensor_init_qpass() {
 }
 
 cudaError_t as_tensor_qpass(const as_launch_args& a, cudaStream_t st) {
+  if (as_tensor_qstream_handles(a)) return as_tensor_qstream(a, st);   // no softmax tokens, the common feature map
   const int BH = a.B * a.H;
   const bool lin = a.n_l > 0;
   CUtensorMap tmQ, tmK, tmV, tmW, tmSt, tmW1, tmO;
