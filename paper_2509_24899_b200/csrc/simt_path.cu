@@ -103,9 +103,20 @@ __global__ void reduce_state_kernel(as_launch_args a) {
   const int bh = blockIdx.y;
   const int D = a.d, F = a.F;
   const int i = blockIdx.x * blockDim.x + threadIdx.x;      // over F*D entries, then F entries of z
+  // (the loads of eight chunks are issued together, the sum still runs in chunk order)
   if (i < F * D) {
+    const float* src = a.part_s + (size_t)bh * a.n_chunks * F * D + i;
+    const size_t pitch = (size_t)F * D;
     float s = 0.f;
-    for (int c = 0; c < a.n_chunks; ++c) s += a.part_s[((size_t)bh * a.n_chunks + c) * F * D + i];
+    int c = 0;
+    for (; c + 8 <= a.n_chunks; c += 8) {
+      float v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = __ldcs(src + (c + j) * pitch);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) s += v[j];
+    }
+    for (; c < a.n_chunks; ++c) s += __ldcs(src + c * pitch);
     a.S[(size_t)bh * F * D + i] = s;
     a.Sb[(size_t)bh * F * D + i] = __float2bfloat16_rn(s);
   } else if (i < F * D + F) {
