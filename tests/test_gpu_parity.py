@@ -531,3 +531,26 @@ def test_many_units_per_cta(mode, name):
     got, got_aux, ref, ref_aux, ex = _run(wl, FULL_PATH, mode, gain)
     assert_parity(got, ref, _tag(name, FULL_PATH, mode, True))
     _check_aux(got_aux, ref_aux, wl, ex["n_softmax"])
+
+
+# Layers without softmax tokens, one-layer map with F = d = 128: the streaming form of the query stage.  The cases
+# cover how its runs of 128-row tiles are dealt to the CTAs: fewer tiles than SMs, heads that get one or two CTAs
+# each, more heads than SMs (runs that cross heads: W and S are replaced on the way), a ragged last tile, degree 1.
+STREAMING = {
+    "few_tiles": W.Workload("s1", B=1, H=2, d=128, F=128, grid=(1, 10, 30), block=(1, 5, 6), rate=0, seed=41),
+    "one_or_two_ctas_per_head": W.Workload("s2", B=2, H=50, d=128, F=128, grid=(1, 10, 25), block=(1, 5, 5), rate=0, seed=42),
+    "more_heads_than_sms_degree1": W.Workload("s3", B=3, H=60, d=128, F=128, grid=(1, 10, 30), block=(1, 5, 6), rate=0, seed=43,
+                                              degree=1),
+    "long_runs": W.Workload("s4", B=1, H=1, d=128, F=128, grid=(8, 30, 52), block=(1, 6, 8), rate=0, seed=44),
+}
+
+
+@pytest.mark.parametrize("name", sorted(STREAMING))
+def test_layers_without_softmax_tokens_streaming_form(name):
+    wl = STREAMING[name]
+    got, got_aux, ref, ref_aux, ex = _run(wl, FULL_PATH, O.STAB_PAPER, want_state=True)
+    assert ex["n_softmax"] == 0
+    ok = np.isfinite(ref).all(-1)          # a query with all-zero features is NaN in both
+    assert ok.mean() > 0.99
+    assert_parity(got[ok], ref[ok], _tag("streaming/" + name, FULL_PATH, O.STAB_PAPER))
+    _check_aux(got_aux[ok], ref_aux[ok], wl, 0)
