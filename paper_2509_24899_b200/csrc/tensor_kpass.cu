@@ -357,7 +357,7 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       bulk_store_1d(p.part_s + (slot * p.F + f) * D, smem_u32(stage), D * 4);
       tma_store_commit();
       p.part_z[slot * p.F + f] = (z0 + z1) + sZ[f_local];
-      tma_store_wait_all();
+      tma_store_wait_read();                                   // the staging rows have been read; the writes land by the end of the kernel
     }
   }
 

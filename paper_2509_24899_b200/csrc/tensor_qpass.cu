@@ -920,7 +920,7 @@ qlin_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     const int n_grp = (n_mine > p.n_rounds && p.split_last && g == 1) ? p.n_rounds : n_mine;
     for (int u = 0; u < n_grp; ++u)
       if (!q_linear_unit<D, GEN>(p, c, &tmO, smem, sDl, u)) break;
-    if ((threadIdx.x & 31) == 0) tma_store_wait_all();
+    if ((threadIdx.x & 31) == 0) tma_store_wait_read();
   }
 
   tc_fence_before();
@@ -993,7 +993,7 @@ qpass_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     const int n_grp = (n_mine > p.n_rounds && p.split_last && warp >= 4) ? p.n_rounds : n_mine;
     for (int u = 0; u < n_grp; ++u)
       if (!q_softmax_unit<D, TWO, GEN>(p, c, &tmO, smem, u)) break;
-    if ((threadIdx.x & 31) == 0) tma_store_wait_all();   // this warp's output stores have completed
+    if ((threadIdx.x & 31) == 0) tma_store_wait_read();  // this warp's output stores have read their rows (the writes land by the end of the kernel)
   }
 
   // ------------------------------------------------------------ teardown

@@ -208,7 +208,7 @@ __device__ __noinline__ void qs_compute(const QSParams& p, const QSCtx& c, const
       ap[0] = 0.f; ap[1] = 0.f; ap[2] = den;
     }
   }
-  if (lane == 0) tma_store_wait_all();               // this warp's output stores have completed
+  if (lane == 0) tma_store_wait_read();              // this warp's output stores have read their rows (the writes land by the end of the kernel)
 }
 
 __global__ void __launch_bounds__(QS_THREADS, 1)
