@@ -565,6 +565,53 @@ def run_stack(args):
     return 0
 
 
+def run_backward(args, wl):
+    """The gradient of the value-distillation loss w.r.t. the feature-map weights ("Attention Distillation"): one
+    forward that keeps its per-row statistics, then backward_phi, device-timed separately.  One JSON line of its
+    own (the headline line is the forward pass); one-layer maps with F = d only."""
+    import torch
+    from paper_2509_24899_b200 import HybridAttention, workloads as W
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; the product path has no CPU fallback")
+    torch.cuda.set_device(0)
+    data = W.generate(wl)
+    dev = {k: torch.from_numpy(v.view("int16")).cuda().view(torch.bfloat16) for k, v in data.items()}
+    y_t = torch.from_numpy(W.teacher_output(wl).view("int16")).cuda().view(torch.bfloat16)
+    op = HybridAttention.from_workload(wl)
+    out = torch.empty_like(dev["q"])
+    aux = torch.empty(wl.B, wl.H, wl.N, 3, dtype=torch.float32, device="cuda")
+
+    def fwd():
+        op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], out=out, aux=aux)
+
+    def bwd():
+        return op.backward_phi(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], y_t, out, aux)
+
+    for _ in range(max(args.warmup, 3)):
+        fwd(); bwd()
+    torch.cuda.synchronize()
+    assert op.last_status() == 0, "device time-out during warm-up"
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    f_ms = b_ms = 0.0
+    for _ in range(args.steps):
+        ev[0].record(); fwd(); ev[1].record(); bwd(); ev[2].record()
+        torch.cuda.synchronize()
+        f_ms += ev[0].elapsed_time(ev[1]); b_ms += ev[1].elapsed_time(ev[2])
+    dwq, dwk, loss = bwd()
+    torch.cuda.synchronize()
+    n_l = wl.N - op.n_softmax
+    # products of the chain rule per head: dphi_q = g' S^T - (g'.y) z (N x d x F), dW_q (N x F x d), dS (N x F x d),
+    # dphi_k = v dS^T + dz (N_L x d x F), dW_k (N_L x F x d); 2 flops per multiply-add
+    flops = wl.B * wl.H * 2.0 * wl.F * wl.d * (3 * wl.N + 2 * n_l)
+    print(json.dumps({"op": "forward(aux) + backward_phi", "metric": "gradient step of the phi weights", "unit": "ms",
+                      "forward_ms": f_ms / args.steps, "backward_ms": b_ms / args.steps, "steps": args.steps,
+                      "backward_gflop": flops / 1e9, "backward_tflops": flops / (b_ms / args.steps * 1e-3) / 1e12,
+                      "loss": float(loss.item()), "grad_norms": [float(dwq.norm()), float(dwk.norm())],
+                      "dtype": "bf16 in, fp32 arithmetic (CUDA cores)", "data": "synthetic",
+                      "config": config_of(wl, op.n_softmax, 1), "device_status": op.last_status()}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -581,6 +628,8 @@ def main():
     ap.add_argument("--shard", default="batch", choices=["batch", "seq"],
                     help="batch: every rank its own layer input (the headline, weak scaling); seq: one layer with its "
                          "tokens spread over the ranks (strong scaling, two NCCL exchanges per layer)")
+    ap.add_argument("--op", default="forward", choices=["forward", "backward"],
+                    help="forward: the headline line; backward: forward with statistics + gradient w.r.t. the phi weights")
     ap.add_argument("--skip-extras", action="store_true",
                     help="only the device-timed steps (for profiler runs): no e2e, no CPU baseline")
     args = ap.parse_args()
@@ -595,6 +644,8 @@ def main():
         wl = W.CONFIGS[args.workload]
     if args.impl == "reference":
         return run_reference(args, wl)
+    if args.op == "backward":
+        return run_backward(args, wl)
     if args.shard == "seq":
         return run_seq_shard(args, wl)
     return run_ours(args, wl)

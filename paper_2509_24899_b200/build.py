@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "lib", "libas_hybrid_attn.so")
-SOURCES = ["as_hybrid_attn.cu", "simt_path.cu", "tensor_init.cu", "tensor_qpass.cu", "tensor_qstream.cu", "tensor_kpass.cu", "backward_simt.cu", "no_alloc.cu",
+SOURCES = ["as_hybrid_attn.cu", "simt_path.cu", "tensor_init.cu", "tensor_qpass.cu", "tensor_qstream.cu", "tensor_kpass.cu", "backward_simt.cu", "backward_tensor.cu", "no_alloc.cu",
            "block_rates.cu"]
 
 

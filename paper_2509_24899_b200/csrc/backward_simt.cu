@@ -1,6 +1,8 @@
 // Gradient of the value-distillation loss L = sum |y - y_hat| ("Attention Distillation", value-distillation
 // loss; Algorithm 1 updates the feature maps only) w.r.t. the feature-map weights W_q, W_k of one hybrid
-// attention layer.  First version: fp32 on CUDA cores, one-layer feature maps with F == d and no bias.
+// attention layer, in fp32 on CUDA cores: one-layer feature maps with F == d and no bias.  (With d = F = 128 on the tensor
+// path the products run on the tensor cores instead, backward_tensor.cu; this file keeps the reductions, the layout
+// of the partial results and the entry points.)
 //
 // With y_hat_i = num_i / den_i, num_i = N_i + lambda_i phi_q,i S, den_i = D_i + lambda_i phi_q,i . z (N_i, D_i: the
 // softmax branch, independent of the weights) the chain rule gives, per (batch, head):
@@ -15,6 +17,7 @@
 #include <algorithm>
 
 #include "as_internal.h"
+#include "backward_common.h"
 
 namespace {
 
@@ -22,16 +25,6 @@ constexpr int BW_THREADS = 512;
 constexpr int BW_TOK = 16;            // tokens per step
 
 __device__ __forceinline__ float bf2f(__nv_bfloat16 x) { return __bfloat162float(x); }
-
-struct BwParams {
-  const __nv_bfloat16 *q, *k, *v, *wq, *wk, *y, *yhat;
-  const float *aux, *S, *z;          // forward results: aux [BH][N][3], S [BH][F][D], z [BH][F]
-  const int32_t* sm_rank;
-  float *part_dS, *part_dz, *part_dW, *part_loss;     // per (bh, chunk)
-  float *dS, *dz;                    // [BH][F][D], [BH][F]
-  float *dWq, *dWk, *loss;           // outputs: [H][F][D] each, one float (may be NULL)
-  int B, H, N, P, n_s, stab_mode, chunks, chunk_tokens;
-};
 
 // phi = r^p and its slope p r^(p-1) for r = relu(a), p = 1 + (index of the feature's part)
 __device__ __forceinline__ void poly(float a, int p, float& phi, float& slope) {
@@ -252,6 +245,7 @@ __global__ void bw_reduce_kernel(BwParams p, int D, int stage) {
       float s = 0.f;
       for (int c = 0; c < p.chunks; ++c) s += p.part_dS[((size_t)bh * p.chunks + c) * F * D + i];
       p.dS[(size_t)bh * F * D + i] = s;
+      p.dSb[(size_t)bh * F * D + i] = __float2bfloat16_rn(s);      // the tensor-core key side's MMA operand
     } else if (i < F * D + F) {
       const int f = i - F * D;
       float s = 0.f;
@@ -279,7 +273,7 @@ __global__ void bw_reduce_kernel(BwParams p, int D, int stage) {
 
 size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
-struct BwLayout { size_t part_dS, part_dz, part_dW, part_loss, dS, dz, total; int chunks, chunk_tokens; };
+struct BwLayout { size_t part_dS, part_dz, part_dW, part_loss, dS, dz, dSb, total; int chunks, chunk_tokens; };
 
 BwLayout bw_layout(const as_hybrid_attn_s* h) {
   const auto& d = h->desc;
@@ -287,9 +281,11 @@ BwLayout bw_layout(const as_hybrid_attn_s* h) {
   BwLayout L{};
   int sms = 148;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
-  const int steps = (d.N + BW_TOK - 1) / BW_TOK;
+  // chunks of whole 128-token tiles (the tensor-core kernels work tile by tile; a multiple of BW_TOK as well)
+  constexpr int STEP = 128;
+  const int steps = (d.N + STEP - 1) / STEP;
   int chunks = std::max(1, std::min(steps, (int)(sms / BH)));
-  L.chunk_tokens = (steps + chunks - 1) / chunks * BW_TOK;
+  L.chunk_tokens = (steps + chunks - 1) / chunks * STEP;
   L.chunks = (d.N + L.chunk_tokens - 1) / L.chunk_tokens;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
@@ -299,6 +295,7 @@ BwLayout bw_layout(const as_hybrid_attn_s* h) {
   L.part_loss = take(BH * L.chunks * 4);
   L.dS = take(BH * F * D * 4);
   L.dz = take(BH * F * 4);
+  L.dSb = take(BH * F * D * 2);
   L.total = off;
   return L;
 }
@@ -350,9 +347,11 @@ as_status_t as_hybrid_attn_backward_phi(as_hybrid_attn_t h, const void* q, const
   p.wq = (const __nv_bfloat16*)w->wq1; p.wk = (const __nv_bfloat16*)w->wk1;
   p.y = (const __nv_bfloat16*)y_teacher; p.yhat = (const __nv_bfloat16*)y_hat;
   p.aux = aux; p.S = (const float*)(fws + h->ws.S); p.z = (const float*)(fws + h->ws.z);
+  p.Sb = (const __nv_bfloat16*)(fws + h->ws.Sb); p.status = h->d_status;
   p.sm_rank = h->d_sm_rank;
   p.part_dS = (float*)(ws + L.part_dS); p.part_dz = (float*)(ws + L.part_dz); p.part_dW = (float*)(ws + L.part_dW);
   p.part_loss = (float*)(ws + L.part_loss); p.dS = (float*)(ws + L.dS); p.dz = (float*)(ws + L.dz);
+  p.dSb = (__nv_bfloat16*)(ws + L.dSb);
   p.dWq = dWq; p.dWk = dWk; p.loss = loss;
   p.B = d.B; p.H = d.H; p.N = d.N; p.P = d.poly_degree; p.n_s = h->n_s; p.stab_mode = d.stab_mode;
   p.chunks = L.chunks; p.chunk_tokens = L.chunk_tokens;
@@ -360,7 +359,13 @@ as_status_t as_hybrid_attn_backward_phi(as_hybrid_attn_t h, const void* q, const
   const int BH = d.B * d.H, D = d.d;
   const dim3 grid(L.chunks, BH), rgrid((D * D + D + 255) / 256, std::max(BH, d.H), 2);
   cudaError_t e = cudaSuccess;
-  if (D == 128) {
+  if (D == 128 && d.phi_dim == 128 && d.kernel_path == AS_PATH_TENSOR) {
+    // the products on the tensor cores; the same fixed-order reductions
+    if ((e = as_bw_tensor_init()) == cudaSuccess && (e = as_bw_tensor_query(p, st)) == cudaSuccess) {
+      bw_reduce_kernel<<<rgrid, 256, 0, st>>>(p, D, 0);
+      if ((e = as_bw_tensor_key(p, st)) == cudaSuccess) bw_reduce_kernel<<<rgrid, 256, 0, st>>>(p, D, 1);
+    }
+  } else if (D == 128) {
     if ((e = cudaFuncSetAttribute(bw_query_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwSmem<128>::BYTES)) == cudaSuccess &&
         (e = cudaFuncSetAttribute(bw_key_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwSmem<128>::BYTES)) == cudaSuccess) {
       bw_query_kernel<128><<<grid, BW_THREADS, BwSmem<128>::BYTES, st>>>(p);

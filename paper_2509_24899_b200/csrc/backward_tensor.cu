@@ -1,0 +1,423 @@
+// Gradient of the value-distillation loss w.r.t. the feature-map weights ("Attention Distillation"; Algorithm 1
+// updates the feature maps only) on the tensor cores, for one-layer maps with d = F = 128 and no bias.  The chain rule
+// (formulas in backward_simt.cu) is a handful of products per 128-token tile:
+//
+//   query side   A  = Q W_q^T                  pre-activations                   [tokens x F]
+//                U  = g S^T                     g = sign(y_hat - y) / den         [tokens x F]
+//                dS  += (lambda phi_q)^T g      state gradient                    [F x d]
+//                dW_q += (dL/da_q)^T Q          dL/da_q = lambda (U + z s) phi'    [F x d]
+//   key side     A  = K W_k^T,  T = V dS^T,     dW_k += (dL/da_k)^T K             dL/da_k = (T + dz) phi' on linear tokens
+//
+// bf16 operands, fp32 accumulation in TMEM.  dz = sum_i lambda phi_q,i s_i is summed, in token order, from the very
+// bf16 values the dS product multiplies (through shared memory).  One CTA per (token chunk, batch*head): sixteen
+// compute warps - a token row (= TMEM lane) is shared by four threads, each taking 32 of its 128 columns - and lane
+// 0 of warp 16, which loads the tiles and issues the products, one tile at a time.  The chunks' partial results leave
+// in the layout of the CUDA-core version and are added up by its fixed-order reduction kernels.  Every wait is
+// bounded (status word, abort flag).
+#include "backward_common.h"
+#include "tensor_common.cuh"
+
+namespace {
+
+using namespace as_tc;
+
+constexpr int BT_COMPUTE = 512;          // warps 0-15: row = thread % 128, column quarter = thread / 128
+constexpr int BT_THREADS = BT_COMPUTE + 32;   // warp 16: TMA + MMA issue (lane 0)
+constexpr int TILE = 128 * 128 * 2;      // bytes of a [128 x 128] bf16 tile
+constexpr uint32_t ID_KK = make_idesc(128, 128, 0, 0);      // both operands K-major
+constexpr uint32_t ID_MM = make_idesc(128, 128, 1, 1);      // both operands MN-major (token rows are the K index)
+
+// barriers (per-tile ones are used once per tile: phase = tile index)
+constexpr int B_WFULL = 0, B_FULL = 1, B_ARDY = 2, B_GRDY = 3, B_URDY = 4, B_PRDY = 5, B_DONE = 6, B_DZ = 7, B_COUNT = 8;
+
+struct BtLayout {
+  static constexpr int W_OFF = 0;                 // weights [F][d]
+  static constexpr int S_OFF = TILE;              // S (query side) / dS (key side) in bf16 [F][d]
+  static constexpr int X_OFF = 2 * TILE;          // Q / K tile
+  static constexpr int Y_OFF = 3 * TILE;          // query side: y, then g in place.  key side: V, then dL/da_k in place
+  static constexpr int H_OFF = 4 * TILE;          // query side: y_hat, then lambda phi_q in place
+  static constexpr int A_OFF = 5 * TILE;          // query side: dL/da_q
+  static constexpr int BAR_OFF = 6 * TILE;
+  static constexpr int SVEC_OFF = BAR_OFF + 128;  // 2 x 4 x 128 floats: the column quarters' shares of G . y_hat, per tile parity
+  static constexpr int ZVEC_OFF = SVEC_OFF + 4096;   // 128 floats: z (query side) / dz (key side)
+  static constexpr int RED_OFF = ZVEC_OFF + 512;  // 512 floats: the token quarters' shares of dz at the end, then the warps' loss sums
+  static constexpr int TOTAL = RED_OFF + 2048 + 1024;   // + slack for the 1024-byte alignment
+};
+
+// phi = r^p and its slope p r^(p-1) for r = relu(a)
+AS_DEV void bt_poly(float a, int p, float& phi, float& slope) {
+  const float r = fmaxf(a, 0.f);
+  float rp1 = 1.f;                                // r^(p-1)
+  for (int i = 1; i < p; ++i) rp1 *= r;
+  phi = rp1 * r;
+  slope = a > 0.f ? (float)p * rp1 : 0.f;
+}
+AS_DEV float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
+AS_DEV float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// Writes 32 columns of one accumulator row (TMEM lane = feature row) to dst.
+AS_DEV void bt_store_acc(uint32_t tacc, float* dst) {
+  uint32_t x[32];
+  tmem_ld32(tacc, x);
+  tmem_ld_wait(x);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) reinterpret_cast<uint4*>(dst)[i] = make_uint4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]);
+}
+
+// ---------------------------------------------------------------------------------------------- query side
+__global__ void __launch_bounds__(BT_THREADS, 1)
+btq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmH,
+           const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmS, const __grid_constant__ BwParams p) {
+  using L = BtLayout;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  auto bar = [&](int i) { return sbase + L::BAR_OFF + 8 * i; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::BAR_OFF + 8 * B_COUNT);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::BAR_OFF + 8 * B_COUNT + 4);
+  float* svec = reinterpret_cast<float*>(smem + L::SVEC_OFF);
+  float* zvec = reinterpret_cast<float*>(smem + L::ZVEC_OFF);
+  float* red = reinterpret_cast<float*>(smem + L::RED_OFF);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = blockIdx.y, chunk = blockIdx.x, h = bh % p.H;
+  const int tok_begin = chunk * p.chunk_tokens;
+  const int tok_end = min(p.N, tok_begin + p.chunk_tokens);
+  const int nt = (tok_end - tok_begin + 127) / 128;
+
+  __shared__ uint32_t s_skip;
+  if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile uint32_t*>(p.status);
+  __syncthreads();
+  if (s_skip != 0u) return;
+  if (threadIdx.x == 0) {
+    *abort_flag = 0u;
+    mbar_init(bar(B_WFULL), 1); mbar_init(bar(B_FULL), 1); mbar_init(bar(B_ARDY), 1); mbar_init(bar(B_GRDY), BT_COMPUTE);
+    mbar_init(bar(B_URDY), 1); mbar_init(bar(B_PRDY), BT_COMPUTE); mbar_init(bar(B_DONE), 1); mbar_init(bar(B_DZ), BT_COMPUTE);
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 16) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tA = tmem, tU = tmem + 128, tdS = tmem + 256, tdW = tmem + 384;
+  const WaitCtx wc{p.status, abort_flag};
+
+  if (warp == 16) {
+    if (lane == 0) {
+      tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmY); tma_prefetch_desc(&tmH);
+      mbar_expect_tx(bar(B_WFULL), 2 * TILE);
+      load_tile<128>(sbase + L::W_OFF, &tmW, bar(B_WFULL), 0, h);
+      load_tile<128>(sbase + L::S_OFF, &tmS, bar(B_WFULL), 0, bh);
+      bool ok = true;
+      for (int t = 0; t < nt && ok; ++t) {
+        // the previous tile's products and its dz pass have read the tiles
+        if (t > 0) ok = mbar_wait(bar(B_DONE), (t - 1) & 1, wc) && mbar_wait(bar(B_DZ), (t - 1) & 1, wc);
+        if (!ok) break;
+        const int row0 = tok_begin + t * 128;
+        mbar_expect_tx(bar(B_FULL), 3 * TILE);
+        load_tile<128>(sbase + L::X_OFF, &tmQ, bar(B_FULL), row0, bh);
+        load_tile<128>(sbase + L::Y_OFF, &tmY, bar(B_FULL), row0, bh);
+        load_tile<128>(sbase + L::H_OFF, &tmH, bar(B_FULL), row0, bh);
+        if (t == 0 && !mbar_wait(bar(B_WFULL), 0, wc)) break;
+        if (!mbar_wait(bar(B_FULL), t & 1, wc)) break;
+        tc_fence_after();
+        issue_kmajor<128>(tA, kmajor_desc(sbase + L::X_OFF), kmajor_desc(sbase + L::W_OFF), ID_KK, false);
+        tc_commit(bar(B_ARDY));
+        if (!mbar_wait(bar(B_GRDY), t & 1, wc)) break;
+        tc_fence_after();
+        issue_kmajor<128>(tU, kmajor_desc(sbase + L::Y_OFF), kmajor_desc(sbase + L::S_OFF), ID_KK, false);
+        tc_commit(bar(B_URDY));
+        if (!mbar_wait(bar(B_PRDY), t & 1, wc)) break;
+        tc_fence_after();
+        const uint64_t aP = mnmajor_desc(sbase + L::H_OFF), bG = mnmajor_desc(sbase + L::Y_OFF);
+        const uint64_t aD = mnmajor_desc(sbase + L::A_OFF), bQ = mnmajor_desc(sbase + L::X_OFF);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) mma_ss(tdS, aP + kstep_mnmajor(kk), bG + kstep_mnmajor(kk), ID_MM, (t > 0 || kk > 0) ? 1u : 0u);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) mma_ss(tdW, aD + kstep_mnmajor(kk), bQ + kstep_mnmajor(kk), ID_MM, (t > 0 || kk > 0) ? 1u : 0u);
+        tc_commit(bar(B_DONE));
+      }
+    }
+    __syncwarp();
+  } else {
+    const int r = threadIdx.x & 127, qt = threadIdx.x >> 7;    // token row of the tile (= TMEM lane) and column quarter
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    const int part = 128 / p.P;
+    if (qt == 0) zvec[r] = p.z[(size_t)bh * 128 + r];
+    named_barrier_sync(1, BT_COMPUTE);
+    float dz_acc = 0.f, loss = 0.f;
+    bool ok = true;
+    uint8_t* sY = smem + L::Y_OFF;
+    uint8_t* sH = smem + L::H_OFF;
+    uint8_t* sA = smem + L::A_OFF;
+    for (int t = 0; t < nt; ++t) {
+      if (ok) ok = mbar_wait_warp(bar(B_FULL), t & 1, wc);
+      const int n = tok_begin + t * 128 + r;
+      const bool in = ok && n < tok_end;
+      float lam = 0.f, den = 1.f;
+      if (in) {
+        const float* ap = p.aux + ((size_t)bh * p.N + n) * 3;
+        lam = (p.stab_mode == AS_STAB_EXACT && p.n_s > 0) ? __expf(-ap[0]) : 1.f;
+        den = ap[1] + lam * ap[2];
+      }
+      const float inv_den = 1.f / den;
+      float* sv = svec + (t & 1) * 512;
+      {
+        // g = sign(y_hat - y) / den over this thread's 32 columns of the row, written over y; its share of G . y_hat
+        // and of the loss on the way
+        float sdot = 0.f;
+        if (ok) {
+#pragma unroll
+          for (int c4 = 0; c4 < 4; ++c4) {
+            const int c = qt * 4 + c4;
+            const uint32_t off = (c >> 3) * BOX_BYTES + swz128_chunk_offset(r, c & 7);
+            const uint4 yv = *reinterpret_cast<const uint4*>(sY + off);
+            const uint4 hv = *reinterpret_cast<const uint4*>(sH + off);
+            const uint32_t yw[4] = {yv.x, yv.y, yv.z, yv.w}, hw[4] = {hv.x, hv.y, hv.z, hv.w};
+            uint32_t gw[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float h0 = bf_lo(hw[i]), h1 = bf_hi(hw[i]);
+              const float d0 = h0 - bf_lo(yw[i]), d1 = h1 - bf_hi(yw[i]);
+              const float G0 = d0 > 0.f ? 1.f : (d0 < 0.f ? -1.f : 0.f), G1 = d1 > 0.f ? 1.f : (d1 < 0.f ? -1.f : 0.f);
+              if (in) { loss += fabsf(d0) + fabsf(d1); sdot += G0 * h0 + G1 * h1; }
+              gw[i] = in ? pack_bf16(G0 * inv_den, G1 * inv_den) : 0u;
+            }
+            *reinterpret_cast<uint4*>(sY + off) = make_uint4(gw[0], gw[1], gw[2], gw[3]);
+          }
+        }
+        sv[qt * 128 + r] = sdot;
+      }
+      fence_proxy_async();
+      mbar_arrive(bar(B_GRDY));
+      if (ok) ok = mbar_wait_warp(bar(B_ARDY), t & 1, wc);
+      if (ok) ok = mbar_wait_warp(bar(B_URDY), t & 1, wc);
+      // (U is complete only after every thread has arrived on the g barrier: the quarters' shares are all there)
+      const float s_i = in ? -((sv[r] + sv[128 + r]) + (sv[256 + r] + sv[384 + r])) * inv_den : 0.f;
+      if (ok) {
+        tc_fence_after();
+        uint32_t xa[32], xu[32];
+        const int cc = qt;                           // this thread's 32 features
+        tmem_ld32(tA + lane_off + cc * 32, xa);
+        tmem_ld32(tU + lane_off + cc * 32, xu);
+        tmem_ld_wait(xa);
+        tmem_ld_wait(xu);
+        const int pw = min((cc * 32) / part, p.P - 1) + 1;            // power of these 32 features
+        uint32_t wp[16], wa[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float ph0, sl0, ph1, sl1;
+          bt_poly(__uint_as_float(xa[2 * i]), pw, ph0, sl0);
+          bt_poly(__uint_as_float(xa[2 * i + 1]), pw, ph1, sl1);
+          const int f = cc * 32 + 2 * i;
+          const float u0 = __uint_as_float(xu[2 * i]) + zvec[f] * s_i, u1 = __uint_as_float(xu[2 * i + 1]) + zvec[f + 1] * s_i;
+          wp[i] = pack_bf16(lam * ph0, lam * ph1);
+          wa[i] = pack_bf16(lam * u0 * sl0, lam * u1 * sl1);
+        }
+        store_row_chunk(sH, r, cc * 32, wp);         // lambda phi_q over y_hat (consumed: every thread is past the g barrier)
+        store_row_chunk(sA, r, cc * 32, wa);
+        tc_fence_before();
+      }
+      fence_proxy_async();
+      mbar_arrive(bar(B_PRDY));
+      // dz[f] += sum over the tile's tokens of (lambda phi)[token][f] * s[token]: feature f = r, tokens of quarter qt
+      named_barrier_sync(1, BT_COMPUTE);             // every row of lambda phi of the tile is in shared memory
+      if (ok) {
+        const uint32_t col = (uint32_t)(r >> 6) * BOX_BYTES + (uint32_t)(r & 7) * 2, chunk8 = (uint32_t)((r & 63) >> 3);
+#pragma unroll 8
+        for (int k = 0; k < 32; ++k) {
+          const int tok = qt * 32 + k;
+          const int ntok = tok_begin + t * 128 + tok;
+          float s_tok = 0.f;
+          if (ntok < tok_end) {
+            // the token's s = -(G . y_hat) / den, from the shares and its denominator
+            const float* ap = p.aux + ((size_t)bh * p.N + ntok) * 3;
+            const float lam_t = (p.stab_mode == AS_STAB_EXACT && p.n_s > 0) ? __expf(-ap[0]) : 1.f;
+            s_tok = -((sv[tok] + sv[128 + tok]) + (sv[256 + tok] + sv[384 + tok])) / (ap[1] + lam_t * ap[2]);
+          }
+          const uint16_t hbits = *reinterpret_cast<const uint16_t*>(sH + col + swz128_chunk_offset(tok, chunk8));
+          dz_acc = fmaf(__uint_as_float((uint32_t)hbits << 16), s_tok, dz_acc);
+        }
+      }
+      mbar_arrive(bar(B_DZ));
+    }
+    // ---- the chunk's partial results
+    if (ok && nt > 0) ok = mbar_wait_warp(bar(B_DONE), (nt - 1) & 1, wc);
+    const size_t slot = (size_t)bh * p.chunks + chunk;
+    if (ok && nt > 0) {
+      tc_fence_after();
+      bt_store_acc(tdS + lane_off + qt * 32, p.part_dS + (slot * 128 + r) * 128 + qt * 32);
+      bt_store_acc(tdW + lane_off + qt * 32, p.part_dW + (slot * 128 + r) * 128 + qt * 32);
+      tc_fence_before();
+    }
+    // dz of the chunk: the four token quarters' shares in quarter order; the loss: the sixteen warps' sums in warp order
+    red[qt * 128 + r] = dz_acc;
+    named_barrier_sync(1, BT_COMPUTE);
+    if (qt == 0) p.part_dz[slot * 128 + r] = (red[r] + red[128 + r]) + (red[256 + r] + red[384 + r]);
+    named_barrier_sync(1, BT_COMPUTE);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, off);
+    if (lane == 0) red[warp] = loss;
+    named_barrier_sync(1, BT_COMPUTE);
+    if (threadIdx.x == 0) {
+      float l = 0.f;
+      for (int w = 0; w < 16; ++w) l += red[w];
+      p.part_loss[slot] = l;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 16) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------- key side
+__global__ void __launch_bounds__(BT_THREADS, 1)
+btk_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmW,
+           const __grid_constant__ CUtensorMap tmS, const __grid_constant__ BwParams p) {
+  using L = BtLayout;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  auto bar = [&](int i) { return sbase + L::BAR_OFF + 8 * i; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::BAR_OFF + 8 * B_COUNT);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::BAR_OFF + 8 * B_COUNT + 4);
+  float* zvec = reinterpret_cast<float*>(smem + L::ZVEC_OFF);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = blockIdx.y, chunk = blockIdx.x, h = bh % p.H;
+  const int tok_begin = chunk * p.chunk_tokens;
+  const int tok_end = min(p.N, tok_begin + p.chunk_tokens);
+  const int nt = (tok_end - tok_begin + 127) / 128;
+
+  __shared__ uint32_t s_skip;
+  if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile uint32_t*>(p.status);
+  __syncthreads();
+  if (s_skip != 0u) return;
+  if (threadIdx.x == 0) {
+    *abort_flag = 0u;
+    mbar_init(bar(B_WFULL), 1); mbar_init(bar(B_FULL), 1); mbar_init(bar(B_ARDY), 1);
+    mbar_init(bar(B_PRDY), BT_COMPUTE); mbar_init(bar(B_DONE), 1);
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 16) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tA = tmem, tT = tmem + 128, tdW = tmem + 256;
+  const WaitCtx wc{p.status, abort_flag};
+
+  if (warp == 16) {
+    if (lane == 0) {
+      tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+      mbar_expect_tx(bar(B_WFULL), 2 * TILE);
+      load_tile<128>(sbase + L::W_OFF, &tmW, bar(B_WFULL), 0, h);
+      load_tile<128>(sbase + L::S_OFF, &tmS, bar(B_WFULL), 0, bh);
+      for (int t = 0; t < nt; ++t) {
+        if (t > 0 && !mbar_wait(bar(B_DONE), (t - 1) & 1, wc)) break;     // the previous tile's last product has read K and dL/da
+        const int row0 = tok_begin + t * 128;
+        mbar_expect_tx(bar(B_FULL), 2 * TILE);
+        load_tile<128>(sbase + L::X_OFF, &tmK, bar(B_FULL), row0, bh);
+        load_tile<128>(sbase + L::Y_OFF, &tmV, bar(B_FULL), row0, bh);
+        if (t == 0 && !mbar_wait(bar(B_WFULL), 0, wc)) break;
+        if (!mbar_wait(bar(B_FULL), t & 1, wc)) break;
+        tc_fence_after();
+        issue_kmajor<128>(tA, kmajor_desc(sbase + L::X_OFF), kmajor_desc(sbase + L::W_OFF), ID_KK, false);
+        issue_kmajor<128>(tT, kmajor_desc(sbase + L::Y_OFF), kmajor_desc(sbase + L::S_OFF), ID_KK, false);
+        tc_commit(bar(B_ARDY));
+        if (!mbar_wait(bar(B_PRDY), t & 1, wc)) break;
+        tc_fence_after();
+        const uint64_t aD = mnmajor_desc(sbase + L::Y_OFF), bK = mnmajor_desc(sbase + L::X_OFF);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) mma_ss(tdW, aD + kstep_mnmajor(kk), bK + kstep_mnmajor(kk), ID_MM, (t > 0 || kk > 0) ? 1u : 0u);
+        tc_commit(bar(B_DONE));
+      }
+    }
+    __syncwarp();
+  } else {
+    const int r = threadIdx.x & 127, qt = threadIdx.x >> 7;
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    const int part = 128 / p.P;
+    if (qt == 0) zvec[r] = p.dz[(size_t)bh * 128 + r];
+    named_barrier_sync(1, BT_COMPUTE);
+    bool ok = true;
+    uint8_t* sV = smem + L::Y_OFF;
+    for (int t = 0; t < nt; ++t) {
+      if (ok) ok = mbar_wait_warp(bar(B_ARDY), t & 1, wc);
+      const int n = tok_begin + t * 128 + r;
+      const bool lin = ok && n < tok_end && p.sm_rank[n] < 0;
+      if (ok) {
+        tc_fence_after();
+        uint32_t xa[32], xt[32];
+        const int cc = qt;                           // this thread's 32 features
+        tmem_ld32(tA + lane_off + cc * 32, xa);
+        tmem_ld32(tT + lane_off + cc * 32, xt);
+        tmem_ld_wait(xa);
+        tmem_ld_wait(xt);
+        const int pw = min((cc * 32) / part, p.P - 1) + 1;
+        uint32_t wa[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float ph0, sl0, ph1, sl1;
+          bt_poly(__uint_as_float(xa[2 * i]), pw, ph0, sl0);
+          bt_poly(__uint_as_float(xa[2 * i + 1]), pw, ph1, sl1);
+          const int f = cc * 32 + 2 * i;
+          const float t0 = (__uint_as_float(xt[2 * i]) + zvec[f]) * sl0, t1 = (__uint_as_float(xt[2 * i + 1]) + zvec[f + 1]) * sl1;
+          wa[i] = lin ? pack_bf16(t0, t1) : 0u;
+        }
+        store_row_chunk(sV, r, cc * 32, wa);         // dL/da_k over v (the product that read v has completed)
+        tc_fence_before();
+      }
+      fence_proxy_async();
+      mbar_arrive(bar(B_PRDY));
+    }
+    if (ok && nt > 0) ok = mbar_wait_warp(bar(B_DONE), (nt - 1) & 1, wc);
+    if (ok && nt > 0) {
+      tc_fence_after();
+      const size_t slot = (size_t)bh * p.chunks + chunk;
+      bt_store_acc(tdW + lane_off + qt * 32, p.part_dW + (slot * 128 + r) * 128 + qt * 32);
+      tc_fence_before();
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 16) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+}  // namespace
+
+cudaError_t as_bw_tensor_init() {
+  cudaError_t e;
+  if ((e = opt_in_smem(btq_kernel, BtLayout::TOTAL)) != cudaSuccess) return e;
+  return opt_in_smem(btk_kernel, BtLayout::TOTAL);
+}
+
+cudaError_t as_bw_tensor_query(const BwParams& p, cudaStream_t st) {
+  const int BH = p.B * p.H;
+  CUtensorMap tmQ, tmY, tmH, tmW, tmS;
+  if (!make_map(&tmQ, p.q, 128, p.N, BH, 128) || !make_map(&tmY, p.y, 128, p.N, BH, 128) ||
+      !make_map(&tmH, p.yhat, 128, p.N, BH, 128) || !make_map(&tmW, p.wq, 128, 128, p.H, 128) ||
+      !make_map(&tmS, p.Sb, 128, 128, BH, 128))
+    return cudaErrorInvalidValue;
+  btq_kernel<<<dim3(p.chunks, BH), BT_THREADS, BtLayout::TOTAL, st>>>(tmQ, tmY, tmH, tmW, tmS, p);
+  return cudaGetLastError();
+}
+
+cudaError_t as_bw_tensor_key(const BwParams& p, cudaStream_t st) {
+  const int BH = p.B * p.H;
+  CUtensorMap tmK, tmV, tmW, tmS;
+  if (!make_map(&tmK, p.k, 128, p.N, BH, 128) || !make_map(&tmV, p.v, 128, p.N, BH, 128) ||
+      !make_map(&tmW, p.wk, 128, 128, p.H, 128) || !make_map(&tmS, p.dSb, 128, 128, BH, 128))
+    return cudaErrorInvalidValue;
+  btk_kernel<<<dim3(p.chunks, BH), BT_THREADS, BtLayout::TOTAL, st>>>(tmK, tmV, tmW, tmS, p);
+  return cudaGetLastError();
+}
