@@ -39,14 +39,17 @@ def _teacher_with_margin(wl, d64, mode, margin=0.05):
     return W.f32_to_bf16_bits(np.nan_to_num(y_hat + off).astype(np.float32))
 
 
-def _run(wl, mode, gain, margin):
+def _run(wl, mode, gain, margin, simt=False):
     import torch
-    from paper_2509_24899_b200 import HybridAttention
+    from paper_2509_24899_b200 import HybridAttention, binding
     data = W.generate(wl, wq_gain=gain)
     y_bits = _teacher_with_margin(wl, oracle_inputs(data), mode) if margin else W.teacher_output(wl)
     dev = {k: to_cuda_bf16(v) for k, v in data.items()}
     y_dev = to_cuda_bf16(y_bits)
-    op = HybridAttention.from_workload(wl, stab_mode=mode)
+    # (with d = F = 128 the default path runs the products on the tensor cores; the fp32 CUDA-core kernels take every
+    # other shape, and d = F = 128 as well when the handle is on the check path)
+    kw = {"kernel_path": binding.AS_PATH_SIMT} if simt else {}
+    op = HybridAttention.from_workload(wl, stab_mode=mode, **kw)
     aux = torch.empty((wl.B, wl.H, wl.N, 3), dtype=torch.float32, device="cuda")
     y_hat = op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], aux=aux)
     dwq, dwk, loss = op.backward_phi(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"], y_dev, y_hat, aux)
@@ -75,6 +78,18 @@ def test_phi_weight_gradients_match_the_oracle(mode, name, margin):
     assert np.abs(ref_q).max() > 0 and np.abs(ref_k).max() > 0
     tol = 5e-3 if margin else 3e-2
     assert eq <= tol and ek <= tol, (eq, ek)
+    assert abs(loss - ref_loss) <= 2e-3 * ref_loss
+
+
+@pytest.mark.parametrize("name", ["ragged_d128", "rate0", "degree1"])
+def test_phi_weight_gradients_on_the_cuda_core_path(name):
+    """d = F = 128 on the fp32 check path (the default path takes these shapes to the tensor cores)."""
+    wl = CASES[name]
+    dwq, dwk, loss, ref_q, ref_k, ref_loss = _run(wl, O.STAB_PAPER, balanced_gain(wl, O.STAB_PAPER), True, simt=True)
+    eq, ek = errors(dwq, ref_q)[0], errors(dwk, ref_k)[0]
+    _record({"case": "backward/%s/paper/teacher-with-margin/cuda-cores" % name, "rel_l2_dWq": eq, "rel_l2_dWk": ek,
+             "loss_rel_err": abs(loss - ref_loss) / ref_loss})
+    assert eq <= 5e-3 and ek <= 5e-3, (eq, ek)
     assert abs(loss - ref_loss) <= 2e-3 * ref_loss
 
 
