@@ -211,9 +211,10 @@ AS_API as_status_t as_hybrid_attn_query_pass(as_hybrid_attn_t h, const void* q, 
  *              without linear tokens, whose gradients are zero)
  *   workspace  device scratch, 256-byte aligned, >= backward_workspace_bytes
  * L = sum |y - y_hat|; q, k, v and y are constants of the step.  lambda_i (AS_STAB_EXACT: exp(-c_i)) and the softmax
- * branch do not depend on the weights.  First version: fp32 on CUDA cores; one-layer feature maps with F == d and
- * no bias, anything else returns AS_ERR_UNSUPPORTED.  Asynchronous on the stream; sums in a fixed order (no float
- * atomics), so results are run-to-run identical. */
+ * branch do not depend on the weights.  One-layer feature maps with F == d and no bias; anything else returns
+ * AS_ERR_UNSUPPORTED.  With d = F = 128 on AS_PATH_TENSOR the products run on the tensor cores (bf16 operands, fp32
+ * accumulation); every other supported shape, and AS_PATH_SIMT, in fp32 on CUDA cores.  Asynchronous on the stream;
+ * sums in a fixed order (no float atomics), so results are run-to-run identical. */
 AS_API as_status_t as_hybrid_attn_backward_workspace_bytes(as_hybrid_attn_t h, size_t* bytes);
 AS_API as_status_t as_hybrid_attn_backward_phi(as_hybrid_attn_t h, const void* q, const void* k, const void* v,
                                                const as_phi_weights_t* w, const void* y_teacher, const void* y_hat,
