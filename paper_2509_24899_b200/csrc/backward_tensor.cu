@@ -28,6 +28,7 @@ constexpr uint32_t ID_KK = make_idesc(128, 128, 0, 0);      // both operands K-m
 constexpr uint32_t ID_MM = make_idesc(128, 128, 1, 1);      // both operands MN-major (token rows are the K index)
 
 // barriers (per-tile ones are used once per tile: phase = tile index)
+constexpr int B_FULL1 = 3;                  // key side: the second K/V set's "full" barrier (the slot of B_GRDY)
 constexpr int B_WFULL = 0, B_FULL = 1, B_ARDY = 2, B_GRDY = 3, B_URDY = 4, B_PRDY = 5, B_DONE = 6, B_DZ = 7, B_COUNT = 8;
 
 struct BtLayout {
@@ -299,7 +300,7 @@ btk_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
   if (s_skip != 0u) return;
   if (threadIdx.x == 0) {
     *abort_flag = 0u;
-    mbar_init(bar(B_WFULL), 1); mbar_init(bar(B_FULL), 1); mbar_init(bar(B_ARDY), 1);
+    mbar_init(bar(B_WFULL), 1); mbar_init(bar(B_FULL), 1); mbar_init(bar(B_FULL1), 1); mbar_init(bar(B_ARDY), 1);
     mbar_init(bar(B_PRDY), BT_COMPUTE); mbar_init(bar(B_DONE), 1);
     fence_barrier_init();
     fence_proxy_async();
@@ -318,24 +319,45 @@ btk_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
       mbar_expect_tx(bar(B_WFULL), 2 * TILE);
       load_tile<128>(sbase + L::W_OFF, &tmW, bar(B_WFULL), 0, h);
       load_tile<128>(sbase + L::S_OFF, &tmS, bar(B_WFULL), 0, bh);
-      for (int t = 0; t < nt; ++t) {
-        if (t > 0 && !mbar_wait(bar(B_DONE), (t - 1) & 1, wc)) break;     // the previous tile's last product has read K and dL/da
-        const int row0 = tok_begin + t * 128;
-        mbar_expect_tx(bar(B_FULL), 2 * TILE);
-        load_tile<128>(sbase + L::X_OFF, &tmK, bar(B_FULL), row0, bh);
-        load_tile<128>(sbase + L::Y_OFF, &tmV, bar(B_FULL), row0, bh);
-        if (t == 0 && !mbar_wait(bar(B_WFULL), 0, wc)) break;
-        if (!mbar_wait(bar(B_FULL), t & 1, wc)) break;
+      // K and V tiles are double-buffered: tile t lives in set t & 1 (its own "full" barrier), and the tile after the
+      // next is requested as soon as the last product that reads the set has completed
+      auto sK = [&](int t) { return sbase + ((t & 1) ? L::H_OFF : L::X_OFF); };
+      auto sVt = [&](int t) { return sbase + ((t & 1) ? L::A_OFF : L::Y_OFF); };
+      auto full = [&](int t) { return bar((t & 1) ? B_FULL1 : B_FULL); };
+      auto request = [&](int t) {
+        mbar_expect_tx(full(t), 2 * TILE);
+        load_tile<128>(sK(t), &tmK, full(t), tok_begin + t * 128, bh);
+        load_tile<128>(sVt(t), &tmV, full(t), tok_begin + t * 128, bh);
+      };
+      auto first_products = [&](int t) {           // A = K W_k^T and T = V dS^T of tile t
         tc_fence_after();
-        issue_kmajor<128>(tA, kmajor_desc(sbase + L::X_OFF), kmajor_desc(sbase + L::W_OFF), ID_KK, false);
-        issue_kmajor<128>(tT, kmajor_desc(sbase + L::Y_OFF), kmajor_desc(sbase + L::S_OFF), ID_KK, false);
+        issue_kmajor<128>(tA, kmajor_desc(sK(t)), kmajor_desc(sbase + L::W_OFF), ID_KK, false);
+        issue_kmajor<128>(tT, kmajor_desc(sVt(t)), kmajor_desc(sbase + L::S_OFF), ID_KK, false);
         tc_commit(bar(B_ARDY));
-        if (!mbar_wait(bar(B_PRDY), t & 1, wc)) break;
+      };
+      bool ok = nt > 0;
+      if (ok) {
+        request(0);
+        if (nt > 1) request(1);
+        ok = mbar_wait(bar(B_WFULL), 0, wc) && mbar_wait(full(0), 0, wc);
+        if (ok) first_products(0);
+      }
+      for (int t = 0; t < nt && ok; ++t) {
+        if (!mbar_wait(bar(B_PRDY), t & 1, wc)) break;                   // dL/da_k of tile t is in shared memory (over V)
         tc_fence_after();
-        const uint64_t aD = mnmajor_desc(sbase + L::Y_OFF), bK = mnmajor_desc(sbase + L::X_OFF);
+        const uint64_t aD = mnmajor_desc(sVt(t)), bK = mnmajor_desc(sK(t));
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) mma_ss(tdW, aD + kstep_mnmajor(kk), bK + kstep_mnmajor(kk), ID_MM, (t > 0 || kk > 0) ? 1u : 0u);
         tc_commit(bar(B_DONE));
+        // the threads have read A and T of tile t (they arrived on the barrier above): the next tile's may land
+        if (t + 1 < nt) {
+          if (!mbar_wait(full(t + 1), ((t + 1) >> 1) & 1, wc)) break;
+          first_products(t + 1);
+        }
+        if (t + 2 < nt) {
+          if (!mbar_wait(bar(B_DONE), t & 1, wc)) break;                 // the set of tile t is free
+          request(t + 2);
+        }
       }
     }
     __syncwarp();
@@ -346,8 +368,8 @@ btk_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
     if (qt == 0) zvec[r] = p.dz[(size_t)bh * 128 + r];
     named_barrier_sync(1, BT_COMPUTE);
     bool ok = true;
-    uint8_t* sV = smem + L::Y_OFF;
     for (int t = 0; t < nt; ++t) {
+      uint8_t* sV = smem + ((t & 1) ? L::A_OFF : L::Y_OFF);      // the V tile of the set tile t lives in
       if (ok) ok = mbar_wait_warp(bar(B_ARDY), t & 1, wc);
       const int n = tok_begin + t * 128 + r;
       const bool lin = ok && n < tok_end && p.sm_rank[n] < 0;
