@@ -41,7 +41,8 @@ struct BtLayout {
   static constexpr int BAR_OFF = 6 * TILE;
   static constexpr int SVEC_OFF = BAR_OFF + 128;  // 2 x 4 x 128 floats: the column quarters' shares of G . y_hat, per tile parity
   static constexpr int ZVEC_OFF = SVEC_OFF + 4096;   // 128 floats: z (query side) / dz (key side)
-  static constexpr int RED_OFF = ZVEC_OFF + 512;  // 512 floats: the token quarters' shares of dz at the end, then the warps' loss sums
+  static constexpr int SROW_OFF = ZVEC_OFF + 512; // 2 x 128 floats: s of the tile's rows, per tile parity
+  static constexpr int RED_OFF = SROW_OFF + 1024; // 512 floats: the token quarters' shares of dz at the end, then the warps' loss sums
   static constexpr int TOTAL = RED_OFF + 2048 + 1024;   // + slack for the 1024-byte alignment
 };
 
@@ -79,6 +80,7 @@ btq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
   float* svec = reinterpret_cast<float*>(smem + L::SVEC_OFF);
   float* zvec = reinterpret_cast<float*>(smem + L::ZVEC_OFF);
   float* red = reinterpret_cast<float*>(smem + L::RED_OFF);
+  float* srow = reinterpret_cast<float*>(smem + L::SROW_OFF);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int bh = blockIdx.y, chunk = blockIdx.x, h = bh % p.H;
   const int tok_begin = chunk * p.chunk_tokens;
@@ -152,15 +154,28 @@ btq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     uint8_t* sY = smem + L::Y_OFF;
     uint8_t* sH = smem + L::H_OFF;
     uint8_t* sA = smem + L::A_OFF;
+    // the row's statistics of the forward pass (c_i, the two parts of the denominator), fetched one tile ahead
+    auto row_stats = [&](int t, float (&a)[3]) {
+      const int n = tok_begin + t * 128 + r;
+      if (t < nt && n < tok_end) {
+        const float* ap = p.aux + ((size_t)bh * p.N + n) * 3;
+        a[0] = ap[0]; a[1] = ap[1]; a[2] = ap[2];
+      } else {
+        a[0] = 0.f; a[1] = 1.f; a[2] = 0.f;
+      }
+    };
+    float st_next[3];
+    row_stats(0, st_next);
     for (int t = 0; t < nt; ++t) {
+      const float st_c[3] = {st_next[0], st_next[1], st_next[2]};
+      row_stats(t + 1, st_next);
       if (ok) ok = mbar_wait_warp(bar(B_FULL), t & 1, wc);
       const int n = tok_begin + t * 128 + r;
       const bool in = ok && n < tok_end;
       float lam = 0.f, den = 1.f;
       if (in) {
-        const float* ap = p.aux + ((size_t)bh * p.N + n) * 3;
-        lam = (p.stab_mode == AS_STAB_EXACT && p.n_s > 0) ? __expf(-ap[0]) : 1.f;
-        den = ap[1] + lam * ap[2];
+        lam = (p.stab_mode == AS_STAB_EXACT && p.n_s > 0) ? __expf(-st_c[0]) : 1.f;
+        den = st_c[1] + lam * st_c[2];
       }
       const float inv_den = 1.f / den;
       float* sv = svec + (t & 1) * 512;
@@ -196,6 +211,7 @@ btq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
       if (ok) ok = mbar_wait_warp(bar(B_URDY), t & 1, wc);
       // (U is complete only after every thread has arrived on the g barrier: the quarters' shares are all there)
       const float s_i = in ? -((sv[r] + sv[128 + r]) + (sv[256 + r] + sv[384 + r])) * inv_den : 0.f;
+      if (qt == 0) srow[(t & 1) * 128 + r] = s_i;    // for the dz pass below (read after the barrier of all compute threads)
       if (ok) {
         tc_fence_after();
         uint32_t xa[32], xu[32];
@@ -226,19 +242,12 @@ btq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
       named_barrier_sync(1, BT_COMPUTE);             // every row of lambda phi of the tile is in shared memory
       if (ok) {
         const uint32_t col = (uint32_t)(r >> 6) * BOX_BYTES + (uint32_t)(r & 7) * 2, chunk8 = (uint32_t)((r & 63) >> 3);
+        const float* st = srow + (t & 1) * 128;
 #pragma unroll 8
         for (int k = 0; k < 32; ++k) {
           const int tok = qt * 32 + k;
-          const int ntok = tok_begin + t * 128 + tok;
-          float s_tok = 0.f;
-          if (ntok < tok_end) {
-            // the token's s = -(G . y_hat) / den, from the shares and its denominator
-            const float* ap = p.aux + ((size_t)bh * p.N + ntok) * 3;
-            const float lam_t = (p.stab_mode == AS_STAB_EXACT && p.n_s > 0) ? __expf(-ap[0]) : 1.f;
-            s_tok = -((sv[tok] + sv[128 + tok]) + (sv[256 + tok] + sv[384 + tok])) / (ap[1] + lam_t * ap[2]);
-          }
           const uint16_t hbits = *reinterpret_cast<const uint16_t*>(sH + col + swz128_chunk_offset(tok, chunk8));
-          dz_acc = fmaf(__uint_as_float((uint32_t)hbits << 16), s_tok, dz_acc);
+          dz_acc = fmaf(__uint_as_float((uint32_t)hbits << 16), st[tok], dz_acc);
         }
       }
       mbar_arrive(bar(B_DZ));
@@ -368,11 +377,14 @@ btk_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
     if (qt == 0) zvec[r] = p.dz[(size_t)bh * 128 + r];
     named_barrier_sync(1, BT_COMPUTE);
     bool ok = true;
+    auto is_linear = [&](int t) { const int n = tok_begin + t * 128 + r; return t < nt && n < tok_end && p.sm_rank[n] < 0; };
+    bool lin_next = is_linear(0);                    // fetched one tile ahead
     for (int t = 0; t < nt; ++t) {
       uint8_t* sV = smem + ((t & 1) ? L::A_OFF : L::Y_OFF);      // the V tile of the set tile t lives in
+      const bool lin_c = lin_next;
+      lin_next = is_linear(t + 1);
       if (ok) ok = mbar_wait_warp(bar(B_ARDY), t & 1, wc);
-      const int n = tok_begin + t * 128 + r;
-      const bool lin = ok && n < tok_end && p.sm_rank[n] < 0;
+      const bool lin = ok && lin_c;
       if (ok) {
         tc_fence_after();
         uint32_t xa[32], xt[32];
