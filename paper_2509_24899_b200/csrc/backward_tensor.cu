@@ -46,13 +46,42 @@ struct BtLayout {
   static constexpr int TOTAL = RED_OFF + 2048 + 1024;   // + slack for the 1024-byte alignment
 };
 
-// phi = r^p and its slope p r^(p-1) for r = relu(a)
-AS_DEV void bt_poly(float a, int p, float& phi, float& slope) {
+// phi = r^p and its slope p r^(p-1) for r = relu(a); the power is a compile-time constant (a thread's 32 features
+// belong to one part of the feature map)
+template <int PW>
+AS_DEV void bt_poly(float a, float& phi, float& slope) {
   const float r = fmaxf(a, 0.f);
   float rp1 = 1.f;                                // r^(p-1)
-  for (int i = 1; i < p; ++i) rp1 *= r;
+#pragma unroll
+  for (int i = 1; i < PW; ++i) rp1 *= r;
   phi = rp1 * r;
-  slope = a > 0.f ? (float)p * rp1 : 0.f;
+  slope = a > 0.f ? (float)PW * rp1 : 0.f;
+}
+// Query side, 32 features of one row: lambda phi_q and dL/da_q = lambda (U + z s) phi' as bf16 pairs.
+template <int PW>
+AS_DEV void bt_q_features(const uint32_t (&xa)[32], const uint32_t (&xu)[32], const float* zv, float s_i, float lam,
+                          uint32_t (&wp)[16], uint32_t (&wa)[16]) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    float ph0, sl0, ph1, sl1;
+    bt_poly<PW>(__uint_as_float(xa[2 * i]), ph0, sl0);
+    bt_poly<PW>(__uint_as_float(xa[2 * i + 1]), ph1, sl1);
+    const float u0 = fmaf(zv[2 * i], s_i, __uint_as_float(xu[2 * i])), u1 = fmaf(zv[2 * i + 1], s_i, __uint_as_float(xu[2 * i + 1]));
+    wp[i] = pack_bf16(lam * ph0, lam * ph1);
+    wa[i] = pack_bf16(lam * u0 * sl0, lam * u1 * sl1);
+  }
+}
+// Key side, 32 features of one row: dL/da_k = (T + dz) phi' on linear tokens, zero on softmax tokens.
+template <int PW>
+AS_DEV void bt_k_features(const uint32_t (&xa)[32], const uint32_t (&xt)[32], const float* zv, bool lin, uint32_t (&wa)[16]) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    float ph0, sl0, ph1, sl1;
+    bt_poly<PW>(__uint_as_float(xa[2 * i]), ph0, sl0);
+    bt_poly<PW>(__uint_as_float(xa[2 * i + 1]), ph1, sl1);
+    const float t0 = (__uint_as_float(xt[2 * i]) + zv[2 * i]) * sl0, t1 = (__uint_as_float(xt[2 * i + 1]) + zv[2 * i + 1]) * sl1;
+    wa[i] = lin ? pack_bf16(t0, t1) : 0u;
+  }
 }
 AS_DEV float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 AS_DEV float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
@@ -196,9 +225,11 @@ btq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             for (int i = 0; i < 4; ++i) {
               const float h0 = bf_lo(hw[i]), h1 = bf_hi(hw[i]);
               const float d0 = h0 - bf_lo(yw[i]), d1 = h1 - bf_hi(yw[i]);
-              const float G0 = d0 > 0.f ? 1.f : (d0 < 0.f ? -1.f : 0.f), G1 = d1 > 0.f ? 1.f : (d1 < 0.f ? -1.f : 0.f);
-              if (in) { loss += fabsf(d0) + fabsf(d1); sdot += G0 * h0 + G1 * h1; }
-              gw[i] = in ? pack_bf16(G0 * inv_den, G1 * inv_den) : 0u;
+              // (rows past the end of the sequence arrive as zeros: no difference, no sign, nothing added)
+              const float G0 = d0 == 0.f ? 0.f : copysignf(1.f, d0), G1 = d1 == 0.f ? 0.f : copysignf(1.f, d1);
+              loss += fabsf(d0) + fabsf(d1);
+              sdot = fmaf(G0, h0, fmaf(G1, h1, sdot));
+              gw[i] = pack_bf16(G0 * inv_den, G1 * inv_den);
             }
             *reinterpret_cast<uint4*>(sY + off) = make_uint4(gw[0], gw[1], gw[2], gw[3]);
           }
@@ -222,15 +253,11 @@ btq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         tmem_ld_wait(xu);
         const int pw = min((cc * 32) / part, p.P - 1) + 1;            // power of these 32 features
         uint32_t wp[16], wa[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float ph0, sl0, ph1, sl1;
-          bt_poly(__uint_as_float(xa[2 * i]), pw, ph0, sl0);
-          bt_poly(__uint_as_float(xa[2 * i + 1]), pw, ph1, sl1);
-          const int f = cc * 32 + 2 * i;
-          const float u0 = __uint_as_float(xu[2 * i]) + zvec[f] * s_i, u1 = __uint_as_float(xu[2 * i + 1]) + zvec[f + 1] * s_i;
-          wp[i] = pack_bf16(lam * ph0, lam * ph1);
-          wa[i] = pack_bf16(lam * u0 * sl0, lam * u1 * sl1);
+        switch (pw) {
+          case 1: bt_q_features<1>(xa, xu, zvec + cc * 32, s_i, lam, wp, wa); break;
+          case 2: bt_q_features<2>(xa, xu, zvec + cc * 32, s_i, lam, wp, wa); break;
+          case 3: bt_q_features<3>(xa, xu, zvec + cc * 32, s_i, lam, wp, wa); break;
+          default: bt_q_features<4>(xa, xu, zvec + cc * 32, s_i, lam, wp, wa); break;
         }
         store_row_chunk(sH, r, cc * 32, wp);         // lambda phi_q over y_hat (consumed: every thread is past the g barrier)
         store_row_chunk(sA, r, cc * 32, wa);
@@ -395,14 +422,11 @@ btk_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
         tmem_ld_wait(xt);
         const int pw = min((cc * 32) / part, p.P - 1) + 1;
         uint32_t wa[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float ph0, sl0, ph1, sl1;
-          bt_poly(__uint_as_float(xa[2 * i]), pw, ph0, sl0);
-          bt_poly(__uint_as_float(xa[2 * i + 1]), pw, ph1, sl1);
-          const int f = cc * 32 + 2 * i;
-          const float t0 = (__uint_as_float(xt[2 * i]) + zvec[f]) * sl0, t1 = (__uint_as_float(xt[2 * i + 1]) + zvec[f + 1]) * sl1;
-          wa[i] = lin ? pack_bf16(t0, t1) : 0u;
+        switch (pw) {
+          case 1: bt_k_features<1>(xa, xt, zvec + cc * 32, lin, wa); break;
+          case 2: bt_k_features<2>(xa, xt, zvec + cc * 32, lin, wa); break;
+          case 3: bt_k_features<3>(xa, xt, zvec + cc * 32, lin, wa); break;
+          default: bt_k_features<4>(xa, xt, zvec + cc * 32, lin, wa); break;
         }
         store_row_chunk(sV, r, cc * 32, wa);         // dL/da_k over v (the product that read v has completed)
         tc_fence_before();
