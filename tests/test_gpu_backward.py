@@ -28,6 +28,8 @@ CASES = {
     "rate0": W.Workload("bw_rate0", B=1, H=2, d=128, F=128, grid=(2, 10, 13), block=(1, 6, 8), rate=0, seed=63),
     "degree1": W.Workload("bw_degree1", B=1, H=2, d=128, F=128, grid=(3, 10, 13), block=(1, 6, 8), rate=3, seed=64, degree=1),
     "degree4_chunks": W.Workload("bw_degree4", B=1, H=1, d=128, F=128, grid=(6, 30, 52), block=(1, 6, 8), rate=8, seed=65, degree=4),
+    # several 128-token tiles per chunk (accumulation across tiles, tiles loaded ahead) and a batch to sum over
+    "tiles_per_chunk_batch": W.Workload("bw_tiles", B=2, H=20, d=128, F=128, grid=(1, 30, 52), block=(1, 6, 8), rate=4, seed=66),
 }
 
 
