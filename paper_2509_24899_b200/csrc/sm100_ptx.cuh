@@ -36,20 +36,6 @@ AS_DEV bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Non-blocking probe of a phase.  mbarrier.try_wait may put the thread to sleep for a while and was measured to
-// return some hundred clocks after the phase had completed; a loop around this probe notices it within a few tens.
-AS_DEV bool mbar_test_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-
 // Bounded wait.  Gives up after about `kWaitLimitCycles` SM clocks (roughly a second), or as soon as
 // another thread of the CTA has given up; then it raises the CTA's abort flag and the global status bit
 // and returns false.  The clock is only looked at every 64 failed polls, so a wait that is satisfied
@@ -78,29 +64,6 @@ AS_DEV bool mbar_wait_limit(uint32_t bar, uint32_t parity, const WaitCtx& w, lon
   return true;
 }
 AS_DEV bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w) { return mbar_wait_limit(bar, parity, w, kWaitLimitCycles); }
-// The same bounded wait as a loop of non-blocking probes, for hand-overs on the critical path of a pipeline whose
-// warps have issue slots to spare: noticing the phase early matters more there than the slots the loop takes.
-AS_DEV bool mbar_spin_wait(uint32_t bar, uint32_t parity, const WaitCtx& w) {
-  if (mbar_test_wait(bar, parity)) return true;
-  long long t0 = 0;
-  uint32_t it = 0;
-  while (!mbar_test_wait(bar, parity)) {
-    if ((++it & 255u) == 0u) {
-      const long long now = clock64();
-      if (t0 == 0) t0 = now;
-      if (*w.abort != 0u || now - t0 > kWaitLimitCycles) {
-        *w.abort = 1u;
-        atomicOr(w.status, 1u);
-        return false;
-      }
-    }
-  }
-  return true;
-}
-AS_DEV bool mbar_spin_wait_warp(uint32_t bar, uint32_t parity, const WaitCtx& w) {
-  const bool ok = mbar_spin_wait(bar, parity, w);
-  return __all_sync(0xffffffffu, ok);
-}
 // Warp-uniform variant: every lane waits, the result is agreed across the warp.
 AS_DEV bool mbar_wait_warp(uint32_t bar, uint32_t parity, const WaitCtx& w) {
   const bool ok = mbar_wait(bar, parity, w);

@@ -95,10 +95,6 @@ AS_DEV int q_units_of_cta(const QParams& p) {
   return p.n_rounds + (extra ? 1 : 0);
 }
 
-// per unit and group: uses of the score columns / releases of the P tile (cf. QRing::n_s, n_pf)
-AS_DEV int q_uses_s(const QParams& p) { return p.nkv + (p.lin ? (p.layers == 2 ? p.nh + p.fc : p.fc) : 0); }
-AS_DEV int q_uses_pf(const QParams& p) { return p.nkv + (p.lin ? (p.layers == 2 ? 1 : p.fc) : 0); }
-
 template <int D>
 struct QRing {
   using L = QLayout<D>;

@@ -51,11 +51,8 @@ struct QSCtx {
   WaitCtx wc;
   long long t0, t1;          // this CTA's tiles [t0, t1)
   AS_DEV uint32_t bar(int i) const { return sbase + QSLayout::BAR_OFF + 8 * i; }
-#ifndef QS_SPIN
-#define QS_SPIN 0
-#endif
-  AS_DEV bool wait(int b, int phase) const { return (QS_SPIN & 2) ? mbar_spin_wait(bar(b), phase & 1, wc) : mbar_wait(bar(b), phase & 1, wc); }
-  AS_DEV bool wait_warp(int b, int phase) const { return (QS_SPIN & 1) ? mbar_spin_wait_warp(bar(b), phase & 1, wc) : mbar_wait_warp(bar(b), phase & 1, wc); }
+  AS_DEV bool wait(int b, int phase) const { return mbar_wait(bar(b), phase & 1, wc); }
+  AS_DEV bool wait_warp(int b, int phase) const { return mbar_wait_warp(bar(b), phase & 1, wc); }
   AS_DEV uint32_t tPhi(int g) const { return tmem + 128u * g; }
   AS_DEV uint32_t tO(int g) const { return tmem + 256u + 128u * g; }
 };
