@@ -197,11 +197,13 @@ as_status_t as_hybrid_attn_create(const as_hybrid_attn_desc_t* desc, as_hybrid_a
   std::vector<int32_t> rank(desc->N, -1);
   for (int i = 0; i < h->n_s; ++i) rank[h->idx_host[i]] = i;
   if (cudaMalloc(&h->d_sm_rank, sizeof(int32_t) * ((size_t)desc->N + 8)) != cudaSuccess ||
-      cudaMalloc(&h->d_status, 256) != cudaSuccess) {
+      cudaMalloc(&h->d_status, 256) != cudaSuccess ||
+      cudaMalloc(&h->d_counters, sizeof(uint32_t) * 8 * (size_t)BH) != cudaSuccess) {
     cudaGetLastError(); as_hybrid_attn_destroy(h); return AS_ERR_ALLOC;
   }
   if (cudaMemcpy(h->d_sm_rank, rank.data(), sizeof(int32_t) * desc->N, cudaMemcpyHostToDevice) != cudaSuccess ||
-      cudaMemset(h->d_status, 0, 256) != cudaSuccess) {
+      cudaMemset(h->d_status, 0, 256) != cudaSuccess ||
+      cudaMemset(h->d_counters, 0, sizeof(uint32_t) * 8 * (size_t)BH) != cudaSuccess) {
     cudaGetLastError(); as_hybrid_attn_destroy(h); return AS_ERR_CUDA;
   }
   if (desc->kernel_path == AS_PATH_TENSOR && as_tensor_init() != cudaSuccess) {
@@ -215,6 +217,7 @@ as_status_t as_hybrid_attn_destroy(as_hybrid_attn_t h) {
   if (!h) return AS_OK;
   if (h->d_sm_rank) cudaFree(h->d_sm_rank);
   if (h->d_status) cudaFree(h->d_status);
+  if (h->d_counters) cudaFree(h->d_counters);
   for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
   for (cudaEvent_t e : h->ev_run) cudaEventDestroy(e);
   if (h->side_ready) {
@@ -305,7 +308,7 @@ static as_status_t launch_heads(as_hybrid_attn_t h, const void* q, const void* k
   a.part_s = (float*)(ws + h->ws.part_s); a.part_z = (float*)(ws + h->ws.part_z);
   a.S = (float*)(ws + h->ws.S) + (size_t)first * F * dd; a.z = (float*)(ws + h->ws.z) + (size_t)first * F;
   a.Sb = (__nv_bfloat16*)(ws + h->ws.Sb) + (size_t)first * F * dd;
-  a.sm_rank = h->d_sm_rank; a.status = h->d_status;
+  a.sm_rank = h->d_sm_rank; a.status = h->d_status; a.counters = h->d_counters;
   a.B = nb; a.H = nh; a.N = d.N; a.d = d.d; a.F = d.phi_dim; a.P = d.poly_degree;
   a.n_s = h->n_s; a.n_l = h->n_l; a.n_chunks = h->n_chunks; a.chunk_tiles = h->chunk_tiles;
   a.scale = h->scale; a.stab_mode = d.stab_mode;
@@ -333,9 +336,12 @@ static as_status_t launch_heads(as_hybrid_attn_t h, const void* q, const void* k
     { ProfileScope p(h, st, AS_KERNEL_KPASS);
       e = simt ? as_simt_kpass(a, st) : as_tensor_kpass(a, st); }
     if (e != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
-    { ProfileScope p(h, st, AS_KERNEL_REDUCE);
-      e = as_reduce_state(a, st); }
-    if (e != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
+    if (simt) {
+      // (the tensor K pass adds the chunks up itself, every CTA of a head a slice, once the head's CTAs have all stored)
+      { ProfileScope p(h, st, AS_KERNEL_REDUCE);
+        e = as_reduce_state(a, st); }
+      if (e != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
+    }
   }
 queries:
   if (!(stages & AS_STAGE_QUERIES)) return AS_OK;
@@ -436,7 +442,11 @@ as_status_t as_hybrid_attn_last_status(as_hybrid_attn_t h, void* cuda_stream) {
       cudaMemcpy(&word, h->d_status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
     cudaGetLastError(); return AS_ERR_CUDA;
   }
-  if (word != 0 && cudaMemset(h->d_status, 0, 4) != cudaSuccess) { cudaGetLastError(); return AS_ERR_CUDA; }
+  // after a time-out CTAs have left early: the K pass's arrival counters may stand anywhere
+  if (word != 0 && (cudaMemset(h->d_status, 0, 4) != cudaSuccess ||
+                    cudaMemset(h->d_counters, 0, sizeof(uint32_t) * 8 * (size_t)h->desc.B * h->desc.H) != cudaSuccess)) {
+    cudaGetLastError(); return AS_ERR_CUDA;
+  }
   return (word & AS_DEV_TIMEOUT) ? AS_ERR_DEVICE_TIMEOUT : AS_OK;
 }
 

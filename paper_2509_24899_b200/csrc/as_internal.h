@@ -39,6 +39,8 @@ struct as_launch_args {
   __nv_bfloat16* Sb;
   const int32_t* sm_rank;               // [N]: position in T_S, or -1 for a linear token
   uint32_t* status;                     // device status word
+  uint32_t* counters;                   // [B*H*4][2], zero between launches: K-pass CTAs of a (batch, head, feature chunk)
+                                        // that have stored their partial state / that have added their slice up
   int B, H, N, d, F, P;
   int n_s, n_l;
   int n_chunks, chunk_tiles;            // K-pass split of the token axis
@@ -54,6 +56,7 @@ struct as_hybrid_attn_s {
   std::vector<int32_t> idx_host;        // sorted T_S
   int32_t* d_sm_rank = nullptr;
   uint32_t* d_status = nullptr;
+  uint32_t* d_counters = nullptr;       // arrival counters of the K pass (cf. as_launch_args::counters)
   int n_chunks = 1, chunk_tiles = 1;
   as_ws_layout ws;
   uint64_t launches = 0;

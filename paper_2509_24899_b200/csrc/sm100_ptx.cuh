@@ -18,6 +18,8 @@ AS_DEV void mbar_init(uint32_t bar, uint32_t count) {
 }
 AS_DEV void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 AS_DEV void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// the same for every state space (global memory written by bulk copies included)
+AS_DEV void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 AS_DEV void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }

@@ -25,6 +25,9 @@ struct KParams {
   const __nv_bfloat16* k;              // two-layer maps gather the softmax K rows from here (no K tile in the ring)
   const __nv_bfloat16* bias;           // last-layer bias [H][F], or nullptr
   float *part_s, *part_z;
+  float *S, *z;                        // [B*H][F][D], [B*H][F]: the chunks' partials added up ...
+  __nv_bfloat16* Sb;                   // ... and S once more rounded to bf16 (the query stage's MMA operand)
+  uint32_t* counters;                  // [B*H][feature chunks][2]: CTAs that have stored / that have added; zero between launches
   uint32_t* status;
 };
 
@@ -357,7 +360,8 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       bulk_store_1d(p.part_s + (slot * p.F + f) * D, smem_u32(stage), D * 4);
       tma_store_commit();
       p.part_z[slot * p.F + f] = (z0 + z1) + sZ[f_local];
-      tma_store_wait_read();                                   // the staging rows have been read; the writes land by the end of the kernel
+      tma_store_wait_all();                                    // the partial state is in global memory ...
+      fence_proxy_async_all();                                 // ... and ordered before what this CTA publishes below
     }
   }
 
@@ -366,6 +370,72 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   if (warp == 9) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
+  }
+  // ---- The chunks' partial states are added up here, in chunk order (fixed order, no float atomics): every CTA of
+  // a (batch, head, feature chunk) takes a slice of the [F x (D + 1)] entries once all of them have stored theirs.
+  // The CTAs of one launch are resident together (one per SM, a cooperative launch when there is more than one
+  // chunk), so the wait ends; it is bounded like every other wait.  The second counter tells the last CTA to finish
+  // its slice that both counters can go back to zero for the next launch.
+  __shared__ uint32_t s_go;
+  uint32_t* cnt = p.counters + 2 * ((size_t)bh * gridDim.z + fc);
+  const uint32_t n_ctas = gridDim.x;
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(cnt, 1u);
+    uint32_t go = 1u, it = 0;
+    long long t0 = 0;
+    while (*reinterpret_cast<volatile uint32_t*>(cnt) < n_ctas) {
+      __nanosleep(100);
+      if ((++it & 63u) == 0u) {
+        const long long now = clock64();
+        if (t0 == 0) t0 = now;
+        if (*abort_flag != 0u || now - t0 > kWaitLimitCycles) { atomicOr(p.status, 1u); go = 0u; break; }
+      }
+      // a CTA that found the status word set never arrives: the others stop waiting as soon as they see it too
+      if (*reinterpret_cast<volatile uint32_t*>(p.status) != 0u) { go = 0u; break; }
+    }
+    s_go = go;
+  }
+  __syncthreads();
+  if (s_go == 0u) return;
+  __threadfence();
+  {
+    const int f0 = fc * 128, nf = min(128, p.F - f0);
+    const size_t pitch = (size_t)p.F * D;                      // floats between two chunks' partials
+    const float* src = p.part_s + ((size_t)bh * p.n_chunks * p.F + f0) * D;
+    float* dS = p.S + ((size_t)bh * p.F + f0) * D;
+    __nv_bfloat16* dSb = p.Sb + ((size_t)bh * p.F + f0) * D;
+    const int n4 = nf * D / 4, per = (n4 + (int)n_ctas - 1) / (int)n_ctas;       // float4 entries, this CTA's slice
+    const int i_end = min(n4, (chunk + 1) * per);
+    for (int i = chunk * per + (int)threadIdx.x; i < i_end; i += K_THREADS) {
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      int c = 0;
+      for (; c + 4 <= p.n_chunks; c += 4) {                    // four chunks' loads in flight, added in chunk order
+        float4 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = __ldcg(reinterpret_cast<const float4*>(src + (c + j) * pitch) + i);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { acc.x += v[j].x; acc.y += v[j].y; acc.z += v[j].z; acc.w += v[j].w; }
+      }
+      for (; c < p.n_chunks; ++c) {
+        const float4 v = __ldcg(reinterpret_cast<const float4*>(src + c * pitch) + i);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      }
+      reinterpret_cast<float4*>(dS)[i] = acc;
+      reinterpret_cast<uint2*>(dSb)[i] = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+    }
+    if (chunk == 0) {
+      for (int f = threadIdx.x; f < nf; f += K_THREADS) {
+        float acc = 0.f;
+        for (int c = 0; c < p.n_chunks; ++c) acc += __ldcg(p.part_z + ((size_t)bh * p.n_chunks + c) * p.F + f0 + f);
+        p.z[(size_t)bh * p.F + f0 + f] = acc;
+      }
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t done = atomicAdd(cnt + 1, 1u);
+    if (done + 1u == n_ctas) { cnt[0] = 0u; cnt[1] = 0u; }     // everyone has read the first counter: ready for the next launch
   }
 }
 
@@ -483,8 +553,14 @@ phi1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUt
 template <int D, int LAYERS, int NH>
 cudaError_t launch_kpass(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmW, const CUtensorMap& tmH,
                          const KParams& p, dim3 grid, cudaStream_t st) {
-  kpass_kernel<D, LAYERS, NH><<<grid, K_THREADS, KLayout<D, LAYERS, NH>::TOTAL, st>>>(tmK, tmV, tmW, tmH, p);
-  return cudaGetLastError();
+  if (grid.x == 1) {                   // one chunk per head: no CTA waits for another
+    kpass_kernel<D, LAYERS, NH><<<grid, K_THREADS, KLayout<D, LAYERS, NH>::TOTAL, st>>>(tmK, tmV, tmW, tmH, p);
+    return cudaGetLastError();
+  }
+  // several chunks per head: the CTAs wait for one another at the end, so they must be resident together
+  void* args[] = {(void*)&tmK, (void*)&tmV, (void*)&tmW, (void*)&tmH, (void*)&p};
+  return cudaLaunchCooperativeKernel((const void*)kpass_kernel<D, LAYERS, NH>, grid, dim3(K_THREADS), args,
+                                     (size_t)KLayout<D, LAYERS, NH>::TOTAL, st);
 }
 
 }  // namespace
@@ -531,6 +607,7 @@ cudaError_t as_tensor_kpass(const as_launch_args& a, cudaStream_t st) {
   p.H = a.H; p.sm_rank = a.sm_rank; p.ks_w = a.ks_w; p.vs_w = a.vs_w; p.k = a.k;
   p.bias = two ? a.bk2 : a.bk1;
   p.part_s = a.part_s; p.part_z = a.part_z; p.status = a.status;
+  p.S = a.S; p.z = a.z; p.Sb = a.Sb; p.counters = a.counters;
   dim3 grid(a.n_chunks, BH, (a.F + 127) / 128);
   if (a.d == 128) {
     if (!two) return launch_kpass<128, 1, 1>(tmK, tmV, tmW, tmH, p, grid, st);

@@ -340,11 +340,12 @@ def test_run_to_run_determinism_and_launch_count():
     b = op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"]).clone()
     torch.cuda.synchronize()
     assert torch.equal(a.view(torch.int16), b.view(torch.int16))
-    assert binding.as_hybrid_attn_launch_count(op.handle) == 6       # K pass, reduce, Q pass; twice
+    # K pass (its CTAs add the chunks' partial states up themselves: no launch of its own) and Q pass; twice
+    assert binding.as_hybrid_attn_launch_count(op.handle) == 4
     binding.as_hybrid_attn_profile_enable(op.handle, True)
     op.forward(dev["q"], dev["k"], dev["v"], dev["wq"], dev["wk"])
     ms, cnt = binding.as_hybrid_attn_profile_read(op.handle)
-    assert cnt == [1, 1, 1] and all(t > 0 for t in ms)
+    assert cnt == [1, 0, 1] and ms[0] > 0 and ms[2] > 0
 
 
 def test_expired_device_wait_is_reported_once_and_the_handle_recovers():
