@@ -140,7 +140,11 @@ AS_API as_status_t as_hybrid_attn_workspace_bytes_host(as_hybrid_attn_t h, size_
  *   workspace device scratch, 256-byte aligned, >= workspace_bytes; contents are overwritten
  *   cuda_stream  a cudaStream_t (NULL = default stream)
  * Enqueues its kernels and returns; errors found on the host are returned at once, a device
- * time-out is reported later by as_hybrid_attn_last_status. */
+ * time-out is reported later by as_hybrid_attn_last_status.  Calls on one handle must be ordered on the device (one
+ * stream, or events between streams): the handle's status word and the arrival counters of the key stage are shared
+ * by its calls.  On AS_PATH_TENSOR the key stage's CTAs wait for one another when a head is cut into several token
+ * chunks, so that kernel is a cooperative launch (at most one CTA per SM): it needs the whole device, and the launch
+ * is refused (AS_ERR_CUDA) where the device cannot hold all of its CTAs at once. */
 AS_API as_status_t as_hybrid_attn_forward(as_hybrid_attn_t h, const void* q, const void* k, const void* v,
                                    const as_phi_weights_t* w, void* out, float* aux,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
