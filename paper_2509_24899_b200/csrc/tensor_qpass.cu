@@ -443,6 +443,55 @@ AS_DEV float q_features_to_tile(const QParams& p, const uint32_t (&ph)[128], uin
   return dl0 + dl1;
 }
 
+// The same for the one-layer tail, 32 columns at a time straight from the score columns (the loop is not unrolled:
+// the tail runs once per unit, and on a CTA's first unit its instructions come from L2 line by line, so its
+// size is its cost).  Arrives on `sf_bar` once the last columns are in registers.
+template <int D, bool GEN>
+AS_DEV float q_features_from_tmem(const QParams& p, uint32_t tSg, uint32_t sf_bar, uint8_t* tile, int r, int bh, int ch, float lam) {
+  const int fcw = D == 128 ? 128 : p.fcw;
+  const int part = p.F / p.P;
+  const float2* zrow = reinterpret_cast<const float2*>(p.z + (size_t)bh * p.F + ch * 128);
+  const uint32_t* brow = nullptr;
+  if (GEN && p.b2 != nullptr) brow = reinterpret_cast<const uint32_t*>(p.b2 + (size_t)(bh % p.H) * p.F + ch * 128);
+  const float2 lam2 = make_float2(lam, lam);
+  float2 dl2 = make_float2(0.f, 0.f);
+  uint32_t x[32];
+#pragma unroll 1
+  for (int cc = 0; cc * 32 < fcw; ++cc) {
+    tmem_ld32(tSg + cc * 32, x);
+    tmem_ld_wait(x);
+    if (cc * 32 + 32 >= fcw) {
+      tc_fence_before();
+      mbar_arrive(sf_bar);                             // the next product into the score columns may follow
+    }
+    const int pw = min((ch * 128 + cc * 32) / part, p.P - 1);     // 0-based part of these 32 features
+    uint32_t wd[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      float a0 = __uint_as_float(x[2 * i]), a1 = __uint_as_float(x[2 * i + 1]);
+      if (GEN && brow != nullptr) {
+        const uint32_t bb = __ldg(brow + cc * 16 + i);            // same address in every lane: one broadcast load
+        a0 += __uint_as_float(bb << 16);
+        a1 += __uint_as_float(bb & 0xffff0000u);
+      }
+      const float2 a = make_float2(fmaxf(a0, 0.f), fmaxf(a1, 0.f));
+      float2 rr = a;
+      if (pw >= 1) rr = __fmul2_rn(rr, a);
+      if (GEN) {
+        if (pw >= 2) rr = __fmul2_rn(rr, a);
+        if (pw >= 3) rr = __fmul2_rn(rr, a);
+      }
+      rr = __fmul2_rn(rr, lam2);
+      wd[i] = pack_bf16(rr.x, rr.y);
+      const float2 zz = __ldg(zrow + cc * 16 + i);
+      dl2 = __ffma2_rn(make_float2(__uint_as_float(wd[i] << 16), __uint_as_float(wd[i] & 0xffff0000u)), zz, dl2);
+    }
+    store_row_chunk(tile, r, cc * 32, wd);
+  }
+  fence_proxy_async();
+  return dl2.x + dl2.y;
+}
+
 // Reads one row of the score columns (ncols of them) at once and releases the columns.
 template <int D>
 AS_DEV void q_read_row(const QRing<D>& q, int g, uint32_t tSg, int ncols, uint32_t (&ph)[128]) {
@@ -684,10 +733,8 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
       for (int ch = 0; ch < q.fc; ++ch) {
         if (!q.wait(R::B_S + g, ps + nkv + ch)) return false;
         tc_fence_after();
-        uint32_t ph[128];                              // this thread's row of Phi: read at once, columns released
-        q_read_row<D>(q, g, tSg, D == 128 ? 128 : p.fcw, ph);
         if (!p_buffer_free(ppf + nkv + ch)) return false;   // the last tile's P V / the previous chunk's product has read the P tile
-        dl += q_features_to_tile<D, GEN>(p, ph, sPg, r, bh, ch, lam);     // phi_q takes P's place as the A operand
+        dl += q_features_from_tmem<D, GEN>(p, tSg, q.bar(R::B_SF + g), sPg, r, bh, ch, lam);   // phi_q takes P's place as the A operand
         mbar_arrive(q.bar(R::B_P + g));
       }
     }
@@ -705,7 +752,7 @@ __device__ __noinline__ bool q_softmax_unit(const QParams& p, const QCtx& c, con
   // The output rows are staged in the group's P tile (the product that read it has completed with the O
   // barrier); each warp stores its own 32 rows (rows past N are clipped by the tensor map).
   const int wrow0 = row - lane;
-#pragma unroll
+#pragma unroll 1
   for (int cc = 0; cc < D / 32; ++cc) {
     tmem_ld32(tOg + cc * 32, x);
     tmem_ld_wait(x);
