@@ -607,7 +607,8 @@ def run_backward(args, wl):
                       "forward_ms": f_ms / args.steps, "backward_ms": b_ms / args.steps, "steps": args.steps,
                       "backward_gflop": flops / 1e9, "backward_tflops": flops / (b_ms / args.steps * 1e-3) / 1e12,
                       "loss": float(loss.item()), "grad_norms": [float(dwq.norm()), float(dwk.norm())],
-                      "dtype": "bf16 in, fp32 arithmetic (CUDA cores)", "data": "synthetic",
+                      "dtype": ("bf16 operands, fp32 accumulation (tcgen05 kernels)" if wl.d == 128 and wl.F == 128
+                                else "bf16 in, fp32 arithmetic (CUDA cores)"), "data": "synthetic",
                       "config": config_of(wl, op.n_softmax, 1), "device_status": op.last_status()}))
     return 0
 
