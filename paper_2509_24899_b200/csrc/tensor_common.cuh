@@ -49,15 +49,18 @@ AS_DEV void issue_tmemA_mnB(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, u
     mma_ts(d_tmem, a_tmem + kk * 8, b_desc + kstep_mnmajor(kk), idesc, (acc || kk > 0) ? 1u : 0u);
 }
 
-// Writes 32 consecutive columns [c0, c0+32) of row `row` of a swizzled [128 x D] bf16 tile.
+// Writes 32 consecutive columns [c0, c0+32) of row `row` of a swizzled [128 x D] bf16 tile (1024-byte aligned).
+// Through a 32-bit shared-memory address and st.shared: the same stores through the generic pointer cost the
+// softmax threads of the Q pass an eighth of their time per key tile.  The row's 16-byte chunk c sits at
+// (row start + ((row & 7) << 4)) ^ (c << 4): one xor per store.
 AS_DEV void store_row_chunk(uint8_t* tile, uint32_t row, uint32_t c0, const uint32_t (&w)[16]) {
-  uint8_t* box = tile + (c0 / 64) * BOX_BYTES;
+  const uint32_t base = smem_u32(tile) + (c0 / 64) * BOX_BYTES + row * 128u + ((row & 7u) << 4);
   const uint32_t chunk0 = (c0 % 64) / 8;
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    uint4 v = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
-    *reinterpret_cast<uint4*>(box + swz128_chunk_offset(row, chunk0 + i)) = v;
-  }
+  for (int i = 0; i < 4; ++i)
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                 ::"r"(base ^ ((chunk0 + i) << 4)), "r"(w[4 * i]), "r"(w[4 * i + 1]), "r"(w[4 * i + 2]), "r"(w[4 * i + 3])
+                 : "memory");
 }
 
 // 3-D bf16 tensor [slices][rows][cols] (cols contiguous) viewed through boxes of 64 cols x box_rows rows
