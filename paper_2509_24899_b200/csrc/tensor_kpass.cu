@@ -84,7 +84,7 @@ kpass_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   using L = KLayout<D, LAYERS, NH>;
   constexpr int SLOTS = L::SLOTS, IPT = L::IPT, NX = L::NX;
   extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t sbase = smem_u32(smem);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::BAR_OFF);
   enum { B_W = 0, B_FULL = 1, B_EMPTY = B_FULL + SLOTS, B_D1 = B_EMPTY + SLOTS, B_PK = B_D1 + 2, B_DONE = B_PK + 2,
@@ -460,7 +460,7 @@ phi1_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUt
             const __grid_constant__ CUtensorMap tmH, const P1Params p) {
   using L = P1Layout<D, NH>;
   extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t sbase = smem_u32(smem);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::BAR_OFF);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::BAR_OFF + 16);

@@ -212,7 +212,7 @@ __global__ void __launch_bounds__(QS_THREADS, 1)
 qstream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmW,
                const __grid_constant__ CUtensorMap tmSt, const __grid_constant__ CUtensorMap tmO, const __grid_constant__ QSParams p) {
   extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t sbase = smem_u32(smem);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + QSLayout::BAR_OFF + 8 * B_COUNT);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + QSLayout::BAR_OFF + 8 * B_COUNT + 4);
