@@ -50,9 +50,9 @@ AS_DEV void issue_tmemA_mnB(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, u
 }
 
 // Writes 32 consecutive columns [c0, c0+32) of row `row` of a swizzled [128 x D] bf16 tile (1024-byte aligned).
-// Through a 32-bit shared-memory address and st.shared: the same stores through the generic pointer cost the
-// softmax threads of the Q pass an eighth of their time per key tile.  The row's 16-byte chunk c sits at
-// (row start + ((row & 7) << 4)) ^ (c << 4): one xor per store.
+// Through a 32-bit shared-memory address and st.shared: run by itself, the Q pass's per-tile instruction stream
+// takes an eighth longer with the same stores issued through the generic pointer.  The row's 16-byte chunk c
+// sits at (row start + ((row & 7) << 4)) ^ (c << 4): one xor per store.
 AS_DEV void store_row_chunk(uint8_t* tile, uint32_t row, uint32_t c0, const uint32_t (&w)[16]) {
   const uint32_t base = smem_u32(tile) + (c0 / 64) * BOX_BYTES + row * 128u + ((row & 7u) << 4);
   const uint32_t chunk0 = (c0 % 64) / 8;
