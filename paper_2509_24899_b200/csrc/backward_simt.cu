@@ -242,8 +242,17 @@ __global__ void bw_reduce_kernel(BwParams p, int D, int stage) {
   const int bh = blockIdx.y;                                    // stage 0, blockIdx.z == 0: per (batch, head)
   if (stage == 0 && blockIdx.z == 0) {
     if (i < F * D) {
+      const float* src = p.part_dS + (size_t)bh * p.chunks * F * D + i;
       float s = 0.f;
-      for (int c = 0; c < p.chunks; ++c) s += p.part_dS[((size_t)bh * p.chunks + c) * F * D + i];
+      int c = 0;
+      for (; c + 4 <= p.chunks; c += 4) {                          // four loads in flight, added in chunk order
+        float v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = __ldcg(src + (size_t)(c + j) * F * D);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) s += v[j];
+      }
+      for (; c < p.chunks; ++c) s += __ldcg(src + (size_t)c * F * D);
       p.dS[(size_t)bh * F * D + i] = s;
       p.dSb[(size_t)bh * F * D + i] = __float2bfloat16_rn(s);      // the tensor-core key side's MMA operand
     } else if (i < F * D + F) {
@@ -260,8 +269,18 @@ __global__ void bw_reduce_kernel(BwParams p, int D, int stage) {
   float* out = stage == 0 ? p.dWq : p.dWk;
   if (i < F * D) {
     float s = 0.f;
-    for (int b = 0; b < p.B; ++b)
-      for (int c = 0; c < p.chunks; ++c) s += p.part_dW[((size_t)(b * p.H + h) * p.chunks + c) * F * D + i];
+    for (int b = 0; b < p.B; ++b) {
+      const float* src = p.part_dW + (size_t)(b * p.H + h) * p.chunks * F * D + i;
+      int c = 0;
+      for (; c + 4 <= p.chunks; c += 4) {                          // four loads in flight, added in (batch, chunk) order
+        float v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = __ldcg(src + (size_t)(c + j) * F * D);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) s += v[j];
+      }
+      for (; c < p.chunks; ++c) s += __ldcg(src + (size_t)c * F * D);
+    }
     out[(size_t)h * F * D + i] = s;
   }
   if (stage == 0 && h == 0 && i == 0 && p.loss != nullptr) {
